@@ -1,0 +1,233 @@
+/*
+ * CPU oracle for the composed-prefill hot path.  TEST INFRASTRUCTURE ONLY:
+ * it is what the CUDA library is checked against and what the bench times as
+ * its CPU baseline; no product code path may call it.
+ *
+ * Plain definitions in fp64, one token / one row at a time, no tiling, no
+ * online softmax, no page skipping.  It shares no code with the CUDA library.
+ *
+ *   oracle_placement      - "placement before preparation" (Sec. 5.3): the request's
+ *                           final KV slots are fixed first; storage blocks of B
+ *                           tokens, ceil(n/B) per unit, not adjacent (Sec. 5.1).
+ *   oracle_rope_rotate    - rotary embedding of one head vector by an angle index
+ *                           delta (Sec. 2.2: queries and keys are rotated, values
+ *                           are not; a cached key is brought to its new offset).
+ *   oracle_assemble       - "preparing cache hits" + "completing prefill" (Sec. 5.3):
+ *                           cached rows placed at request positions with keys
+ *                           rotated to the new positions; recomputed rows private
+ *                           to the request override cached ones.
+ *   oracle_attention_rows - the extend pass restricted to the recompute rows
+ *                           (Sec. 5.3, Sec. 6.1 "Implementation"): causal softmax
+ *                           attention of a query at position p over keys 0..p.
+ *
+ * Pins (tests/test_oracle_pins.py): composition and relative-position identities,
+ * one-hot closed form, a library rotary routine, a 2-D rotation matrix, the
+ * paper's worked position example, brute-force attention, library causal
+ * attention, uniform-softmax closed form, per-token placement loop.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double bf16_to_double(uint16_t b) {
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* -------------------------------------------------------------------------
+ * Placement (Sec. 5.3 "Placement before preparation"; Sec. 5.1 storage blocks).
+ * Request r takes the next ceil(T_r / B) ids of free_pages, in batch order.
+ * src_slot[p] = pool slot (page * B + offset) holding the cached row that lands
+ * at position p, -1 when no cached unit covers p.  fresh_idx[p] = index into the
+ * recompute list when p is recomputed, else -1.
+ * Returns 0, or a negative number for a batch that has no valid layout.
+ * ------------------------------------------------------------------------- */
+int oracle_placement(int batch, const int32_t *seq_len, const int32_t *unit_off,
+                     const int32_t *unit_len, const int32_t *unit_target_pos,
+                     const int32_t *unit_page_off, const int32_t *unit_pages,
+                     const int32_t *recompute_off, const int32_t *recompute_pos,
+                     const int32_t *free_pages, int n_free, int page_size,
+                     int32_t *page_off, int32_t *pages, int32_t *src_slot, int32_t *fresh_idx)
+{
+    int next_free = 0;
+    long tok_base = 0;
+    page_off[0] = 0;
+    for (int r = 0; r < batch; ++r) {
+        int T = seq_len[r];
+        int need = (T + page_size - 1) / page_size;
+        if (next_free + need > n_free) return -1;
+        for (int k = 0; k < need; ++k) pages[page_off[r] + k] = free_pages[next_free + k];
+        next_free += need;
+        page_off[r + 1] = page_off[r] + need;
+        for (int p = 0; p < T; ++p) { src_slot[tok_base + p] = -1; fresh_idx[tok_base + p] = -1; }
+        for (int u = unit_off[r]; u < unit_off[r + 1]; ++u) {
+            int cached = unit_page_off[u + 1] > unit_page_off[u];
+            for (int i = 0; i < unit_len[u]; ++i) {
+                int p = unit_target_pos[u] + i;
+                if (p < 0 || p >= T) return -2;
+                if (!cached) continue;
+                if (src_slot[tok_base + p] != -1) return -3;            /* two units on one position */
+                src_slot[tok_base + p] = unit_pages[unit_page_off[u] + i / page_size] * page_size + i % page_size;
+            }
+        }
+        for (int j = recompute_off[r]; j < recompute_off[r + 1]; ++j) {
+            int p = recompute_pos[j];
+            if (p < 0 || p >= T) return -4;
+            if (j > recompute_off[r] && recompute_pos[j - 1] >= p) return -5;
+            fresh_idx[tok_base + p] = j;
+        }
+        for (int p = 0; p < T; ++p)
+            if (src_slot[tok_base + p] < 0 && fresh_idx[tok_base + p] < 0) return -6;   /* nobody supplies p */
+        tok_base += T;
+    }
+    return 0;
+}
+
+/* -------------------------------------------------------------------------
+ * Rotary embedding of one head vector by delta positions (Sec. 2.2).
+ * Pair m has frequency w_m = theta^(-2m/D) (or inv_freq[m] when given).
+ * pairing 0: pair m = (x[m], x[m + D/2]); pairing 1: pair m = (x[2m], x[2m+1]).
+ * (a, b) -> (a cos(delta w) - b sin(delta w),  b cos(delta w) + a sin(delta w)).
+ * ------------------------------------------------------------------------- */
+void oracle_rope_rotate(const double *x, double *out, int D, double delta, double theta,
+                        const double *inv_freq, int pairing)
+{
+    int half = D / 2;
+    for (int m = 0; m < half; ++m) {
+        double w = inv_freq ? inv_freq[m] : pow(theta, -2.0 * (double)m / (double)D);
+        double ang = delta * w;
+        double c = cos(ang), s = sin(ang);
+        int ia = pairing ? 2 * m : m;
+        int ib = pairing ? 2 * m + 1 : m + half;
+        double a = x[ia], b = x[ib];
+        out[ia] = a * c - b * s;
+        out[ib] = b * c + a * s;
+    }
+}
+
+/* -------------------------------------------------------------------------
+ * Assembled K and V of request r (Sec. 5.3 "Preparing cache hits", "Completing
+ * prefill").  For every position p < T:
+ *   recomputed position j  -> K = k_new[j], V = v_new[j] (bit copies);
+ *   otherwise, cached unit u at offset i = p - target_pos(u):
+ *        V = pool row (bit copy: values carry no rotation),
+ *        K = pool row rotated by delta = p - (cached_pos(u) + stride(u) * i).
+ * k_asm is fp64 and left unrounded.  k_bits / k_exact: rows whose result is a bit
+ * copy (recomputed rows and delta == 0) are given as bf16 bits with k_exact = 1.
+ * ------------------------------------------------------------------------- */
+int oracle_assemble(int r, const int32_t *seq_len, const int32_t *unit_off,
+                    const int32_t *unit_len, const int32_t *unit_cached_pos,
+                    const int32_t *unit_cached_stride, const int32_t *unit_target_pos,
+                    const int32_t *unit_page_off, const int32_t *unit_pages,
+                    const int32_t *recompute_off, const int32_t *recompute_pos,
+                    int page_size, int H_kv, int D, double theta, const double *inv_freq, int pairing,
+                    const uint16_t *k_pool, const uint16_t *v_pool,
+                    const uint16_t *k_new, const uint16_t *v_new,
+                    double *k_asm, uint16_t *v_asm, uint16_t *k_bits, uint8_t *k_exact, int32_t *delta_out)
+{
+    int T = seq_len[r];
+    size_t row = (size_t)H_kv * D;
+    uint8_t *have = (uint8_t *)calloc((size_t)T + 1, 1);
+    double *tmp = (double *)malloc(sizeof(double) * D);
+    for (int p = 0; p < T; ++p) { k_exact[p] = 0; delta_out[p] = 0; }
+    for (int u = unit_off[r]; u < unit_off[r + 1]; ++u) {
+        if (unit_page_off[u + 1] <= unit_page_off[u]) continue;
+        for (int i = 0; i < unit_len[u]; ++i) {
+            int p = unit_target_pos[u] + i;
+            size_t slot = (size_t)unit_pages[unit_page_off[u] + i / page_size] * page_size + i % page_size;
+            int delta = p - (unit_cached_pos[u] + unit_cached_stride[u] * i);
+            delta_out[p] = delta;
+            memcpy(v_asm + (size_t)p * row, v_pool + slot * row, row * sizeof(uint16_t));
+            for (int h = 0; h < H_kv; ++h) {
+                const uint16_t *src = k_pool + slot * row + (size_t)h * D;
+                double *dst = k_asm + (size_t)p * row + (size_t)h * D;
+                for (int d = 0; d < D; ++d) tmp[d] = bf16_to_double(src[d]);
+                oracle_rope_rotate(tmp, dst, D, (double)delta, theta, inv_freq, pairing);
+            }
+            if (delta == 0) {
+                k_exact[p] = 1;
+                memcpy(k_bits + (size_t)p * row, k_pool + slot * row, row * sizeof(uint16_t));
+            }
+            have[p] = 1;
+        }
+    }
+    for (int j = recompute_off[r]; j < recompute_off[r + 1]; ++j) {
+        int p = recompute_pos[j];
+        memcpy(v_asm + (size_t)p * row, v_new + (size_t)j * row, row * sizeof(uint16_t));
+        memcpy(k_bits + (size_t)p * row, k_new + (size_t)j * row, row * sizeof(uint16_t));
+        for (size_t e = 0; e < row; ++e) k_asm[(size_t)p * row + e] = bf16_to_double(k_new[(size_t)j * row + e]);
+        k_exact[p] = 1;
+        delta_out[p] = 0;
+        have[p] = 1;
+    }
+    int missing = 0;
+    for (int p = 0; p < T; ++p) missing += !have[p];
+    free(have);
+    free(tmp);
+    return missing ? -1 : 0;
+}
+
+/* -------------------------------------------------------------------------
+ * Attention rows (Sec. 5.3 "Completing prefill").  Row i is query token row_q[i]
+ * (index into q [n_q][H_q][D]) with head row_h[i] at position row_pos[i]; it
+ * reads kv head row_h[i] / g (g = H_q / H_kv):
+ *     s_t = scale * <q, K[t]>            t = 0 .. pos
+ *     O   = sum_t softmax(s)_t V[t]
+ *     LSE = log sum_t exp(s_t)
+ * ------------------------------------------------------------------------- */
+void oracle_attention_rows(int T, int H_q, int H_kv, int D, double scale,
+                           const double *k_asm, const uint16_t *v_asm, const uint16_t *q,
+                           int n_rows, const int32_t *row_q, const int32_t *row_h, const int32_t *row_pos,
+                           double *out, double *lse)
+{
+    int g = H_q / H_kv;
+    size_t row = (size_t)H_kv * D;
+    (void)T;
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int i = 0; i < n_rows; ++i) {
+        int h = row_h[i], kvh = h / g, p = row_pos[i];
+        const uint16_t *qv = q + ((size_t)row_q[i] * H_q + h) * D;
+        double *qd = (double *)malloc(sizeof(double) * D);
+        double *s = (double *)malloc(sizeof(double) * ((size_t)p + 1));
+        for (int d = 0; d < D; ++d) qd[d] = bf16_to_double(qv[d]);
+        double mx = -INFINITY;
+        for (int t = 0; t <= p; ++t) {
+            const double *kv = k_asm + (size_t)t * row + (size_t)kvh * D;
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d) acc += qd[d] * kv[d];
+            s[t] = acc * scale;
+            if (s[t] > mx) mx = s[t];
+        }
+        double denom = 0.0;
+        for (int t = 0; t <= p; ++t) { s[t] = exp(s[t] - mx); denom += s[t]; }
+        double *o = out + (size_t)i * D;
+        for (int d = 0; d < D; ++d) o[d] = 0.0;
+        for (int t = 0; t <= p; ++t) {
+            const uint16_t *vv = v_asm + (size_t)t * row + (size_t)kvh * D;
+            double w = s[t] / denom;
+            for (int d = 0; d < D; ++d) o[d] += w * bf16_to_double(vv[d]);
+        }
+        lse[i] = mx + log(denom);
+        free(qd);
+        free(s);
+    }
+}
+
+int oracle_num_threads(void)
+{
+    int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+    {
+#pragma omp master
+        n = omp_get_num_threads();
+    }
+#endif
+    return n;
+}

@@ -1,0 +1,324 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests touches the CUDA library.  Each one is chosen so that a
+plausible slip in the oracle (wrong sign, wrong pairing, wrong frequency, an
+off-by-one in the causal limit, a transposed head mapping, a wrong slot) fails it.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import tessera_oracle as orc
+from paper_2609_32999_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# --------------------------------------------------------------------------- RoPE
+
+@pytest.mark.parametrize("D,theta", [(64, 1e4), (128, 5e5), (8, 100.0)])
+def test_rope_composition(D, theta):
+    """R(d) R(p) k == R(p + d) k, including negative d and d == 0."""
+    rng = np.random.default_rng(1)
+    for p, d in [(0, 17), (100, -100), (150, -100), (31999, 1025), (12, 0), (7, -7), (5, -9)]:
+        k = rng.standard_normal(D)
+        a = orc.rope_rotate(orc.rope_rotate(k, p, theta), d, theta)
+        b = orc.rope_rotate(k, p + d, theta)
+        assert np.max(np.abs(a - b)) < 1e-10
+    k = rng.standard_normal(D)
+    assert np.array_equal(orc.rope_rotate(k, 0, theta), k)
+
+
+def test_rope_relative_position_invariance():
+    """<R(m) q, R(n) k> == <q, R(n - m) k>."""
+    rng = np.random.default_rng(2)
+    D, theta = 128, 5e5
+    for m, n in [(3, 10), (1000, 4), (0, 0), (511, 33023)]:
+        q, k = rng.standard_normal(D), rng.standard_normal(D)
+        lhs = orc.rope_rotate(q, m, theta) @ orc.rope_rotate(k, n, theta)
+        rhs = q @ orc.rope_rotate(k, n - m, theta)
+        assert abs(lhs - rhs) < 1e-9
+
+
+def test_rope_one_hot_closed_form():
+    """k = e_m (first half) -> cos(p w_m) at m, +sin(p w_m) at m + D/2, zero elsewhere;
+    k = e_{m + D/2} -> -sin at m, cos at m + D/2.  Fixes direction, pairing, frequency."""
+    D, theta, p = 16, 10000.0, 5
+    for m in range(D // 2):
+        w = 1.0 / (theta ** (2.0 * m / D))
+        e = np.zeros(D); e[m] = 1.0
+        r = orc.rope_rotate(e, p, theta)
+        exp = np.zeros(D); exp[m] = math.cos(p * w); exp[m + D // 2] = math.sin(p * w)
+        assert np.allclose(r, exp, atol=1e-14)
+        e = np.zeros(D); e[m + D // 2] = 1.0
+        r = orc.rope_rotate(e, p, theta)
+        exp = np.zeros(D); exp[m] = -math.sin(p * w); exp[m + D // 2] = math.cos(p * w)
+        assert np.allclose(r, exp, atol=1e-14)
+    # the first pair turns by exactly p radians (w_0 = 1), the last by p * theta^-(D-2)/D
+    e = np.zeros(D); e[0] = 1.0
+    assert abs(orc.rope_rotate(e, 1, theta)[D // 2] - math.sin(1.0)) < 1e-15
+
+
+def test_rope_2d_is_rotation_matrix():
+    """D = 2: a single pair with w = 1 -> the 2-D counter-clockwise rotation matrix."""
+    for ang in [0.3, -1.2, 2.0]:
+        R = np.array([[math.cos(ang), -math.sin(ang)], [math.sin(ang), math.cos(ang)]])
+        v = np.array([0.7, -1.9])
+        assert np.allclose(orc.rope_rotate(v, ang, 12345.0), R @ v, atol=1e-15)
+
+
+def test_rope_preserves_pair_norms():
+    rng = np.random.default_rng(3)
+    D = 64
+    k = rng.standard_normal(D)
+    r = orc.rope_rotate(k, 977, 1e4)
+    assert np.allclose(k[:32] ** 2 + k[32:] ** 2, r[:32] ** 2 + r[32:] ** 2, atol=1e-12)
+
+
+def test_rope_matches_library_rotary():
+    """Same numbers as the rotary routine of the model family the paper serves
+    (half-split pairing, rotate_half convention), evaluated in fp64."""
+    from transformers.models.llama.modeling_llama import apply_rotary_pos_emb
+    D, theta = 128, 5e5
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal((1, 1, 6, D))                       # [batch, heads, seq, D]
+    pos = np.array([0, 1, 17, 511, 4096, 33023], dtype=np.float64)
+    inv = 1.0 / (theta ** (np.arange(0, D, 2, dtype=np.float64) / D))
+    fr = np.outer(pos, inv)
+    emb = np.concatenate([fr, fr], axis=-1)
+    cos, sin = torch.from_numpy(np.cos(emb))[None], torch.from_numpy(np.sin(emb))[None]
+    xt = torch.from_numpy(x)
+    q_emb, _ = apply_rotary_pos_emb(xt, xt, cos, sin)
+    for i, p in enumerate(pos):
+        ours = orc.rope_rotate(x[0, 0, i], p, theta)
+        assert np.max(np.abs(ours - q_emb[0, 0, i].numpy())) < 1e-10   # angle ulp at 3e4 rad
+
+
+def test_rope_explicit_inv_freq_and_interleaved():
+    D, theta = 32, 1e4
+    rng = np.random.default_rng(5)
+    k = rng.standard_normal(D)
+    inv = theta ** (-2.0 * np.arange(D // 2) / D)
+    assert np.allclose(orc.rope_rotate(k, 9, theta), orc.rope_rotate(k, 9, 1.0, inv_freq=inv), atol=1e-14)
+    # interleaved pairing is the half-split rotation on a permuted vector
+    perm = np.concatenate([np.arange(0, D, 2), np.arange(1, D, 2)])
+    a = orc.rope_rotate(k, 9, theta, pairing=1)
+    b = orc.rope_rotate(k[perm], 9, theta, pairing=0)
+    assert np.allclose(a[perm], b, atol=1e-14)
+
+
+def test_paper_position_example_negative_shift():
+    """Sec. 2.2's example: a document cached at 150-249 reused at 50-149 needs a
+    shift of -100 on every key; shifting equals rotating the raw key at the target."""
+    row = [l for l in open(os.path.join(GOLDEN, "fig1_doc_b_positions.txt")) if not l.startswith("#")][0]
+    c0, c1, t0, t1 = map(int, row.split())
+    assert c1 - c0 == t1 - t0 == 99 and t0 - c0 == -100
+    shape = wl.ModelShape(2, 1, 16, 16, 10000.0)
+    rng = np.random.default_rng(6)
+    w = wl.build_workload("docB", shape,
+                          [[t0, wl.unit(c1 - c0 + 1, "B", cached_pos=c0), 3]], rng)
+    t = wl.make_tensors(w)
+    kp = orc.bits(t.k_pool).copy()
+    a0 = orc.assemble(w, 0, kp, orc.bits(t.v_pool), orc.bits(t.k_new), orc.bits(t.v_new))
+    assert set(a0.delta[t0:t1 + 1]) == {-100}
+    # independent check of the values: unrotate pool content by its cached position, rotate at target
+    st, page_off, pages, src_slot, fresh = orc.placement(w)
+    assert st == 0
+    pool = orc.bf16_bits_to_f64(kp).reshape(-1, 1, 16)
+    for p in (t0, t0 + 37, t1):
+        i = p - t0
+        cached = pool[src_slot[p], 0]
+        raw_key = orc.rope_rotate(cached, -(c0 + i), 10000.0)
+        direct = orc.rope_rotate(raw_key, p, 10000.0)
+        assert np.max(np.abs(direct - a0.k[p, 0])) < 1e-10
+
+
+# ---------------------------------------------------------------------- placement
+
+def _placement_by_hand(w):
+    """Per-token restatement used only here: walk every unit token by token."""
+    B = w.shape.page_size
+    src = []
+    for r in range(w.batch):
+        s = [-1] * int(w.seq_len[r])
+        for u in range(w.unit_off[r], w.unit_off[r + 1]):
+            pg = w.unit_pages[w.unit_page_off[u]:w.unit_page_off[u + 1]]
+            if len(pg) == 0:
+                continue
+            for i in range(w.unit_len[u]):
+                page, off = divmod(i, B)
+                s[w.unit_target_pos[u] + i] = int(pg[page]) * B + off
+        src.extend(s)
+    return np.array(src, np.int32)
+
+
+@pytest.mark.parametrize("make", [lambda: wl.config(1), lambda: wl.config(2), lambda: wl.adversarial(),
+                                  lambda: wl.config(3, requests_override=3)])
+def test_placement(make):
+    w = make()
+    st, page_off, pages, src_slot, fresh = orc.placement(w)
+    assert st == 0
+    B = w.shape.page_size
+    need = [-(-int(t) // B) for t in w.seq_len]
+    assert list(np.diff(page_off)) == need
+    assert np.array_equal(pages, w.free_pages[: sum(need)])          # consumed in order
+    assert np.array_equal(src_slot, _placement_by_hand(w))
+    # every position has exactly one supplier class and recompute indices are a bijection
+    assert np.all((src_slot >= 0) | (fresh >= 0))
+    assert sorted(fresh[fresh >= 0]) == list(range(w.n_q))
+    # destination pages never alias source pages
+    assert not (set(pages.tolist()) & set(w.unit_pages.tolist()))
+
+
+def test_placement_rejects_bad_batches():
+    shape = wl.ModelShape(2, 1, 16, 16, 1e4)
+    rng = np.random.default_rng(0)
+    w = wl.build_workload("gap", shape, [[4, wl.unit(20, "a"), 2]], rng)
+    w.recompute_pos = w.recompute_pos[1:].copy()                      # position 0 now uncovered
+    w.recompute_off = np.array([0, len(w.recompute_pos)], np.int32)
+    assert orc.placement(w)[0] < 0
+    w = wl.build_workload("few", shape, [[4, wl.unit(20, "a"), 2]], rng)
+    w.free_pages = w.free_pages[:1].copy()
+    assert orc.placement(w)[0] < 0
+    w = wl.build_workload("overlap", shape, [[wl.unit(20, "a"), wl.unit(20, "b")]], rng)
+    w.unit_target_pos = np.array([0, 10], np.int32)
+    assert orc.placement(w)[0] < 0
+
+
+# ---------------------------------------------------------------------- attention
+
+def _tiny(seed=11, D=8):
+    shape = wl.ModelShape(4, 2, D, 4, 100.0)
+    rng = np.random.default_rng(seed)
+    segs = [3, wl.unit(9, "a", cached_pos=2, recompute=(0, 4)), wl.unit(6, "b", cached=False),
+            wl.unit(7, "c", cached_pos=0, stride=0, recompute=(6,)), 4]
+    return wl.build_workload("tiny", shape, [segs], rng)
+
+
+def test_attention_brute_force_tiny():
+    """Triple loop written here from the definition, on T = 29, D = 8."""
+    w = _tiny()
+    t = wl.make_tensors(w, seed=99)
+    kb, vb, qb, knb, vnb = (orc.bits(x) for x in (t.k_pool, t.v_pool, t.q, t.k_new, t.v_new))
+    asm, out, lse = orc.full_layer(w, kb, vb, qb, knb, vnb)
+    a = asm[0]
+    V = orc.bf16_bits_to_f64(a.v_bits)
+    Q = orc.bf16_bits_to_f64(qb)
+    D, g = 8, 2
+    for j, p in enumerate(w.recompute_pos):
+        for h in range(4):
+            s = [sum(Q[j, h, d] * a.k[t_, h // g, d] for d in range(D)) / math.sqrt(D) for t_ in range(p + 1)]
+            z = sum(math.exp(x) for x in s)
+            for d in range(D):
+                o = sum(math.exp(s[t_]) / z * V[t_, h // g, d] for t_ in range(p + 1))
+                assert abs(o - out[j, h, d]) < 1e-12
+            assert abs(math.log(z) - lse[j, h]) < 1e-12
+
+
+def test_partial_equals_rows_of_library_causal_attention():
+    """Recompute set = all tokens reproduces ordinary causal prefill (library SDPA,
+    fp64, KV heads repeated g times); any subset equals the matching rows."""
+    shape = wl.ModelShape(4, 2, 16, 8, 1e4)
+    rng = np.random.default_rng(21)
+    T = 45
+    w_full = wl.build_workload("full", shape, [[wl.unit(T, "a", cached=False)]], rng)
+    t = wl.make_tensors(w_full, seed=5)
+    bits5 = [orc.bits(x) for x in (t.k_pool, t.v_pool, t.q, t.k_new, t.v_new)]
+    _, out, lse = orc.full_layer(w_full, *bits5)
+    Q = torch.from_numpy(orc.bf16_bits_to_f64(bits5[2])).permute(1, 0, 2)[None]         # [1,H,T,D]
+    K = torch.from_numpy(orc.bf16_bits_to_f64(bits5[3])).permute(1, 0, 2).repeat_interleave(2, 0)[None]
+    V = torch.from_numpy(orc.bf16_bits_to_f64(bits5[4])).permute(1, 0, 2).repeat_interleave(2, 0)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(Q, K, V, is_causal=True)[0].permute(1, 0, 2).numpy()
+    assert np.max(np.abs(ref - out)) < 1e-12
+    # a partial mask over the same assembled KV: cached rows hold exactly k_new/v_new content
+    sel = [0, 3, 4, 17, 44]
+    a_k = orc.bf16_bits_to_f64(bits5[3])
+    o2, l2 = orc.attention_rows(w_full, a_k, bits5[4], bits5[2],
+                                np.repeat(sel, 4), np.tile(np.arange(4), len(sel)), np.repeat(sel, 4))
+    assert np.max(np.abs(o2.reshape(len(sel), 4, 16) - ref[sel])) < 1e-12
+    assert np.max(np.abs(l2.reshape(len(sel), 4) - lse[sel])) < 1e-12
+
+
+def test_uniform_softmax_closed_form_and_causal_limit():
+    """K == 0 -> LSE = ln(p + 1) exactly and O = mean of V[0..p]; with V[t, :, 0] = t this
+    is p / 2: any off-by-one in the causal limit or a wrong kv head shows."""
+    w = wl.config(1)
+    sh = w.shape
+    T = int(w.seq_len[0])
+    k = np.zeros((T, sh.num_kv_heads, sh.head_dim))
+    vt = torch.zeros(T, sh.num_kv_heads, sh.head_dim)
+    vt[:, 0, 0] = torch.arange(T, dtype=torch.float32)
+    vt[:, 1, 0] = -2 * torch.arange(T, dtype=torch.float32)
+    vb = orc.bits(vt.to(torch.bfloat16))                 # integers below 512 are exact in bf16? no: use check
+    V = orc.bf16_bits_to_f64(vb)
+    t = wl.make_tensors(w)
+    jj, hh, pp = orc.request_rows(w, 0)
+    o, l = orc.attention_rows(w, k, vb, orc.bits(t.q), jj, hh, pp)
+    g = sh.num_q_heads // sh.num_kv_heads
+    for i in range(len(jj)):
+        p = pp[i]
+        assert abs(l[i] - math.log(p + 1)) < 1e-12
+        assert abs(o[i, 0] - V[: p + 1, hh[i] // g, 0].mean()) < 1e-9
+
+
+def test_needle_inside_and_outside_causal_limit():
+    """One key with an overwhelming logit: it must dominate when at position <= p and be
+    invisible at position p + 1."""
+    shape = wl.ModelShape(1, 1, 8, 4, 1e4)
+    rng = np.random.default_rng(8)
+    T = 23
+    w = wl.build_workload("needle", shape, [[wl.unit(T, "a", cached=False)]], rng)
+    qf = torch.zeros(T, 1, 8); qf[:, 0, 0] = 8.0
+    for needle in (9, 10, 11, 12):
+        kf = torch.zeros(T, 1, 8); kf[needle, 0, 0] = 64.0
+        vf = torch.zeros(T, 1, 8); vf[needle, 0, 1] = 1.0
+        o, _ = orc.attention_rows(w, kf.double().numpy(), orc.bits(vf.to(torch.bfloat16)),
+                                  orc.bits(qf.to(torch.bfloat16)), [10], [0], [10])
+        if needle <= 10:
+            assert o[0, 1] > 0.999999
+        else:
+            assert o[0, 1] == 0.0
+
+
+def test_assemble_precedence_and_exact_rows():
+    """Recomputed rows override cached rows; delta == 0 rows and V rows are bit copies."""
+    w = wl.adversarial()
+    t = wl.make_tensors(w, seed=3)
+    kb, vb, qb, knb, vnb = (orc.bits(x) for x in (t.k_pool, t.v_pool, t.q, t.k_new, t.v_new))
+    st, page_off, pages, src_slot, fresh = orc.placement(w)
+    assert st == 0
+    base = 0
+    row = w.shape.num_kv_heads * w.shape.head_dim
+    kflat, vflat = kb.reshape(-1, row), vb.reshape(-1, row)
+    saw_zero_delta = saw_negative = False
+    for r in range(w.batch):
+        a = orc.assemble(w, r, kb, vb, knb, vnb)
+        T = int(w.seq_len[r])
+        for p in range(T):
+            j, s = fresh[base + p], src_slot[base + p]
+            if j >= 0:
+                assert a.k_exact[p]
+                assert np.array_equal(a.k_bits[p].ravel(), knb[j].ravel())
+                assert np.array_equal(a.v_bits[p].ravel(), vnb[j].ravel())
+            else:
+                assert np.array_equal(a.v_bits[p].ravel(), vflat[s])
+                if a.delta[p] == 0:
+                    saw_zero_delta = True
+                    assert a.k_exact[p] and np.array_equal(a.k_bits[p].ravel(), kflat[s])
+                    assert np.array_equal(a.k[p].ravel(), orc.bf16_bits_to_f64(kflat[s]))
+                saw_negative |= a.delta[p] < 0
+        base += T
+    assert saw_zero_delta and saw_negative
+
+
+def test_kv_byte_model_closed_form():
+    """Sec. 2.4: 2 L (H_kv/TP) d_h w; the paper's example (64 layers, 8 KV heads, d_h 128,
+    16-bit) is 64 KiB per token per rank at TP = 4 ... and 256 KiB summed over 4 ranks."""
+    assert wl.kv_bytes_per_token(64, 8, 128, 2, tp=4) * 4 == 256 * 1024
+    assert wl.kv_bytes_per_token(1, 8, 128, 2) == 4096
+    w = wl.config(2)
+    assert w.total_tokens == 5312 and w.n_q == 352 and w.cached_tokens == 5120
+    assert wl.gather_bytes(w) == 5120 * 8192
