@@ -1,0 +1,194 @@
+/*
+ * tessera.h - C ABI of the composed-prefill hot path on one B200 (sm_100a).
+ *
+ * The path is the per-layer GPU work of a prompt whose context units already
+ * have cached KV (Sec. 5.3 of the paper, "Coordinated Request Execution"):
+ *
+ *   placement  -> tessera_plan_create          (host, once per batch)
+ *   gather     -> tessera_kv_compose           (device, per layer)
+ *   RoPE shift -> tessera_rope_shift           (device, per layer; normally fused into compose)
+ *   attention  -> tessera_partial_prefill_attn (device, per layer)
+ *
+ * Conventions
+ *   - Every function returns a tessera_status (0 = OK, negative = error).  A failed call
+ *     launches nothing and leaves the pool untouched; tessera_last_error() gives the text
+ *     of the calling thread's last failure.  Nothing throws, aborts or traps.
+ *   - "host" / "device" beside a pointer says where the memory lives.  The caller owns every
+ *     buffer it passes; host arrays may be freed as soon as the call returns.  The library owns
+ *     only the opaque plan (its host tables, device tables and staging buffers).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Device
+ *     work is enqueued on it and the call returns without waiting, unless stated otherwise.
+ *   - All K/V/Q/O tensors are bf16 (2 bytes, raw bits), indices are int32.
+ *   - KV pool layout (one K pool and one V pool per layer, same page ids in every layer):
+ *         [num_pool_pages][page_size][num_kv_heads][head_dim]   bf16, contiguous,
+ *     i.e. a page is a storage block of page_size tokens (Sec. 5.1) and one token's row over all
+ *     KV heads is contiguous.  Slot id = page * page_size + offset.  Base pointers must be
+ *     16-byte aligned.
+ */
+#ifndef TESSERA_H_
+#define TESSERA_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define TESSERA_API __attribute__((visibility("default")))
+#else
+#define TESSERA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum tessera_status {
+    TESSERA_OK = 0,
+    TESSERA_INVALID_ARG = -1,          /* null pointer, negative size, malformed CSR arrays        */
+    TESSERA_UNSORTED_POSITIONS = -2,   /* recompute_pos not strictly ascending inside a request     */
+    TESSERA_UNIT_OVERLAP = -3,         /* two cached units claim one position, or a unit leaves [0,T) */
+    TESSERA_UNCOVERED_POSITION = -4,   /* a position has neither a cached unit nor a recompute entry */
+    TESSERA_PAGE_OUT_OF_RANGE = -5,    /* page id outside [0, num_pool_pages), or dest == source    */
+    TESSERA_OUT_OF_PAGES = -6,         /* free_pages too short for the batch                        */
+    TESSERA_UNSUPPORTED_SHAPE = -7,    /* head_dim / page_size / head counts outside the kernels' range */
+    TESSERA_CUDA_ERROR = -8,           /* a CUDA runtime or driver call failed; see tessera_last_error */
+    TESSERA_DEVICE_TIMEOUT = -9        /* a bounded wait inside a kernel gave up (tessera_plan_status) */
+} tessera_status;
+
+/* Model-side constants of one attention layer. */
+typedef struct tessera_model_cfg {
+    int32_t num_q_heads;        /* H_q                                                        */
+    int32_t num_kv_heads;       /* H_kv, divides H_q; query head h reads KV head h / (H_q/H_kv) */
+    int32_t head_dim;           /* D: 64 or 128                                               */
+    int32_t page_size;          /* tokens per storage block, a multiple of 8, at most 128      */
+    double  rope_theta;         /* pair m turns by theta^(-2m/D) per position                  */
+    const double *inv_freq;     /* host, optional [D/2]: overrides rope_theta when non-null     */
+    int32_t rope_pairing;       /* 0 = pair (m, m + D/2); other values: TESSERA_UNSUPPORTED_SHAPE */
+    float   sm_scale;           /* softmax scale; 0 means 1/sqrt(D)                             */
+} tessera_model_cfg;
+
+/*
+ * One batch of composed prompts: the outcome of the paper's per-unit plan (Sec. 5.1) as the
+ * generation node sees it - an ORDERED list of context units per request, where each one was
+ * cached, where it lands, and which positions are recomputed (Sec. 5.3).  All arrays on the host.
+ */
+typedef struct tessera_compose_desc {
+    int32_t batch;
+    const int32_t *seq_len;             /* [batch] composed length T_r                              */
+    const int32_t *unit_off;            /* [batch+1] CSR into the unit arrays                        */
+    const int32_t *unit_len;            /* [n_units] tokens                                          */
+    const int32_t *unit_cached_pos;     /* [n_units] position of the unit's token 0 when cached       */
+    const int32_t *unit_cached_stride;  /* [n_units] 1: key i was cached rotated at cached_pos + i;
+                                                     0: keys were cached before rotation             */
+    const int32_t *unit_target_pos;     /* [n_units] position of token 0 in this prompt               */
+    const int32_t *unit_page_off;       /* [n_units+1] CSR into unit_pages; an empty range marks an
+                                           uncached unit, all of whose tokens must be recomputed      */
+    const int32_t *unit_pages;          /* source page ids, ceil(len/page_size) per cached unit       */
+    const int32_t *recompute_off;       /* [batch+1] CSR into recompute_pos                           */
+    const int32_t *recompute_pos;       /* query rows: positions, strictly ascending per request      */
+    const int32_t *free_pages;          /* destination page ids, consumed in order, request by request */
+    int32_t n_free;
+} tessera_compose_desc;
+
+typedef struct tessera_plan tessera_plan;
+
+enum { TESSERA_PLAN_HOST_ONLY = 1u };   /* plan_create flag: build and validate host tables only,
+                                           touch no device (the plan then serves only the two
+                                           inspection calls below and plan_destroy)               */
+enum { TESSERA_FUSE_ROPE = 1u };        /* kv_compose flag: rotate keys while copying them        */
+
+typedef struct tessera_plan_info {
+    int64_t total_tokens;       /* sum of T_r                                                   */
+    int64_t n_q;                /* recompute rows                                               */
+    int64_t cached_tokens;      /* rows moved by kv_compose                                     */
+    int64_t qk_pairs;           /* sum over query rows of (position + 1)                        */
+    int64_t gather_bytes;       /* cached_tokens * H_kv * D * 2 bytes * 2 (K,V) * 2 (read,write) */
+    int64_t attn_flops;         /* 4 * D * H_q * qk_pairs                                       */
+    int32_t n_rope_rows;        /* distinct shift amounts in the cos/sin table                  */
+    int32_t n_gather_items;     /* thread blocks of the gather kernel                           */
+    int32_t n_attn_items;       /* (q tile, kv head) work items of the attention kernel         */
+    int32_t attn_kernel;        /* 0 = generic SIMT kernel, 1 = tcgen05 kernel                  */
+} tessera_plan_info;
+
+/*
+ * Placement before preparation (Sec. 5.3): fixes every request's layout and its final KV slots.
+ * Validates the batch, hands request r the next ceil(T_r/page_size) ids of free_pages, derives the
+ * per-position source slot, the copy list, the table of shift amounts (cos/sin evaluated in fp64,
+ * stored fp32) and the attention work list, and uploads them on `stream`.  The plan depends on the
+ * layout only, so one plan serves every layer of the batch.
+ *   num_pool_pages: pages in each pool tensor.   flags: 0 or TESSERA_PLAN_HOST_ONLY.
+ * Returns the plan in *out; errors: every code above except DEVICE_TIMEOUT.
+ */
+TESSERA_API int32_t tessera_plan_create(const tessera_model_cfg *cfg, const tessera_compose_desc *desc,
+                            int32_t num_pool_pages, uint32_t flags, tessera_plan **out, void *stream);
+
+/* Frees host and device tables.  The caller must have synchronised every stream that used the plan. */
+TESSERA_API int32_t tessera_plan_destroy(tessera_plan *plan);
+
+/*
+ * Host views of the placement result, valid until plan_destroy: page_off [batch+1], pages (the
+ * request's block table, in position order), src_slot [sum T_r] (pool slot whose cached row lands at
+ * each position, -1 where no cached unit covers it).  Any out pointer may be NULL.
+ */
+TESSERA_API int32_t tessera_plan_block_table(const tessera_plan *plan, const int32_t **page_off,
+                                 const int32_t **pages, const int32_t **src_slot);
+
+TESSERA_API int32_t tessera_plan_get_info(const tessera_plan *plan, tessera_plan_info *info);
+
+/*
+ * Reads the plan's device status word (synchronises `stream` first).  0 when no kernel of this plan
+ * hit a bounded-wait limit since the last call; otherwise TESSERA_DEVICE_TIMEOUT and *detail (host,
+ * nullable) receives a code naming the wait.  The word is cleared by the call.
+ */
+TESSERA_API int32_t tessera_plan_status(tessera_plan *plan, int32_t *detail, void *stream);
+
+/*
+ * Preparing cache hits, on-GPU part (Sec. 5.3): copies every cached unit's K and V token rows from
+ * its source pages into the request's destination pages at the unit's target offset.  V rows are bit
+ * copies (values carry no rotation, Sec. 2.2).  With TESSERA_FUSE_ROPE the K rows are rotated from
+ * their cached position to their new position on the way (fp32 math, one round-to-nearest-even to
+ * bf16; a shift of 0 is a bit copy); without it K rows are bit copies and tessera_rope_shift must
+ * follow.  k_pool, v_pool: device, layout above; source and destination pages live in the same pool.
+ */
+TESSERA_API int32_t tessera_kv_compose(const tessera_plan *plan, void *k_pool, void *v_pool, uint32_t flags, void *stream);
+
+/*
+ * "Applying RoPE to the keys at their new positions" (Sec. 5.3; the fused placement kernel of
+ * Sec. 6.1) as a call of its own: rotates, in place, the destination-page K rows of every cached
+ * unit by (new position - cached position).  NOT idempotent: call exactly once after a compose
+ * without TESSERA_FUSE_ROPE, never after a fused compose.
+ */
+TESSERA_API int32_t tessera_rope_shift(const tessera_plan *plan, void *k_pool, void *stream);
+
+/*
+ * Completing prefill (Sec. 5.3): the extend pass restricted to the recompute rows.
+ *   1. writes k_new / v_new (device, [n_q][H_kv][D], keys already rotated at their target
+ *      positions) into the rows' destination slots, overriding cached values - recomputed states
+ *      belong to this request only.  Skipped when k_new and v_new are both NULL.
+ *   2. out[j][h] = softmax(sm_scale * q[j][h] . K[0..p_j][h/g]) . V[0..p_j][h/g] over the request's
+ *      assembled pages, p_j = recompute_pos[j]; bf16 inputs, fp32 accumulation and softmax.
+ *   q, out: device [n_q][H_q][D] bf16.  lse: device [n_q][H_q] fp32 natural-log sum of exponentials,
+ *   nullable.
+ */
+TESSERA_API int32_t tessera_partial_prefill_attn(const tessera_plan *plan, void *k_pool, void *v_pool,
+                                     const void *q, const void *k_new, const void *v_new,
+                                     void *out, float *lse, void *stream);
+
+/*
+ * The whole per-layer path for callers whose activations live in HOST memory: copies q, k_new,
+ * v_new (host, pinned for full speed) to staging buffers owned by the plan, runs fused compose and
+ * attention, copies out (and lse when non-null) back to the host and waits for `stream`.
+ * The pools stay on the device: they are the resident KV cache.
+ */
+TESSERA_API int32_t tessera_composed_prefill_host(tessera_plan *plan, void *k_pool, void *v_pool,
+                                      const void *q_host, const void *k_new_host, const void *v_new_host,
+                                      void *out_host, float *lse_host, void *stream);
+
+/* Copies the calling thread's last error text into buf (host); returns its length. */
+TESSERA_API int32_t tessera_last_error(char *buf, int32_t len);
+
+/* Kernels this library has launched in this process so far (all plans, all streams). */
+TESSERA_API int64_t tessera_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TESSERA_H_ */

@@ -1,0 +1,280 @@
+// extern "C" boundary: argument checks, plan upload, kernel launches on the caller's stream.
+#include <atomic>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include <cuda_runtime.h>
+
+#include "launch.h"
+#include "plan.h"
+
+namespace tessera {
+
+namespace {
+thread_local std::string g_last_error;
+std::atomic<int64_t> g_launches{0};
+
+int32_t set_error(int32_t code, const std::string &msg) {
+    g_last_error = msg;
+    return code;
+}
+
+int32_t cuda_fail(cudaError_t e, const char *what) {
+    return set_error(TESSERA_CUDA_ERROR, std::string(what) + ": " + cudaGetErrorName(e) + " (" + cudaGetErrorString(e) + ")");
+}
+
+#define TS_CUDA(call)                                       \
+    do {                                                    \
+        cudaError_t e_ = (call);                            \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
+    } while (0)
+
+size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
+
+template <class T>
+size_t place(size_t &off, size_t n) {
+    size_t o = off;
+    off = align_up(off + n * sizeof(T));
+    return o;
+}
+
+int32_t upload(tessera_plan *pl, cudaStream_t st) {
+    using namespace tessera;
+    DeviceTables &d = pl->dev;
+    TS_CUDA(cudaGetDevice(&pl->device));
+    size_t off = 0;
+    const size_t o_src = place<int32_t>(off, pl->g_src.size());
+    const size_t o_dst = place<int32_t>(off, pl->g_dst.size());
+    const size_t o_items = place<GatherItem>(off, pl->items.size());
+    const size_t o_rope = place<float>(off, pl->rope_table.size());
+    const size_t o_fresh = place<int32_t>(off, pl->fresh_dst.size());
+    const size_t o_qpos = place<int32_t>(off, pl->recompute_pos.size());
+    const size_t o_qreq = place<int32_t>(off, pl->q_req.size());
+    const size_t o_poff = place<int32_t>(off, pl->page_off.size());
+    const size_t o_pages = place<int32_t>(off, pl->pages.size());
+    const size_t o_tiles = place<AttnTile>(off, pl->tiles.size());
+    const size_t o_order = place<int32_t>(off, pl->tile_order.size());
+    const size_t o_status = place<int32_t>(off, 4);
+    pl->host_blob.assign(off, 0);
+    char *hb = pl->host_blob.data();
+    auto put = [&](size_t o, const void *src, size_t bytes) { if (bytes) std::memcpy(hb + o, src, bytes); };
+    put(o_src, pl->g_src.data(), pl->g_src.size() * 4);
+    put(o_dst, pl->g_dst.data(), pl->g_dst.size() * 4);
+    put(o_items, pl->items.data(), pl->items.size() * sizeof(GatherItem));
+    put(o_rope, pl->rope_table.data(), pl->rope_table.size() * 4);
+    put(o_fresh, pl->fresh_dst.data(), pl->fresh_dst.size() * 4);
+    put(o_qpos, pl->recompute_pos.data(), pl->recompute_pos.size() * 4);
+    put(o_qreq, pl->q_req.data(), pl->q_req.size() * 4);
+    put(o_poff, pl->page_off.data(), pl->page_off.size() * 4);
+    put(o_pages, pl->pages.data(), pl->pages.size() * 4);
+    put(o_tiles, pl->tiles.data(), pl->tiles.size() * sizeof(AttnTile));
+    put(o_order, pl->tile_order.data(), pl->tile_order.size() * 4);
+    TS_CUDA(cudaMalloc(&d.blob, off));
+    TS_CUDA(cudaMemcpyAsync(d.blob, hb, off, cudaMemcpyHostToDevice, st));
+    char *db = static_cast<char *>(d.blob);
+    d.g_src = reinterpret_cast<int32_t *>(db + o_src);
+    d.g_dst = reinterpret_cast<int32_t *>(db + o_dst);
+    d.items = reinterpret_cast<GatherItem *>(db + o_items);
+    d.rope = reinterpret_cast<float2 *>(db + o_rope);
+    d.fresh_dst = reinterpret_cast<int32_t *>(db + o_fresh);
+    d.q_pos = reinterpret_cast<int32_t *>(db + o_qpos);
+    d.q_req = reinterpret_cast<int32_t *>(db + o_qreq);
+    d.page_off = reinterpret_cast<int32_t *>(db + o_poff);
+    d.pages = reinterpret_cast<int32_t *>(db + o_pages);
+    d.tiles = reinterpret_cast<AttnTile *>(db + o_tiles);
+    d.tile_order = reinterpret_cast<int32_t *>(db + o_order);
+    d.status = reinterpret_cast<int32_t *>(db + o_status);
+    return TESSERA_OK;
+}
+
+int32_t check_device_plan(const tessera_plan *pl) {
+    if (!pl) return set_error(TESSERA_INVALID_ARG, "null plan");
+    if (pl->host_only) return set_error(TESSERA_INVALID_ARG, "plan was created with TESSERA_PLAN_HOST_ONLY");
+    return TESSERA_OK;
+}
+
+bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
+
+int32_t attention(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, const void *k_new,
+                  const void *v_new, void *out, float *lse, cudaStream_t st) {
+    TS_CUDA(launch_scatter_fresh(pl, k_pool, v_pool, k_new, v_new, st));
+    if (pl->attn_kernel == 1) {
+        std::string err;
+        cudaError_t e = launch_attn_tc(pl, k_pool, v_pool, q, out, lse, st, &err);
+        if (e != cudaSuccess) return set_error(TESSERA_CUDA_ERROR, "tcgen05 attention launch: " + err + " / " + cudaGetErrorString(e));
+    } else {
+        TS_CUDA(launch_attn_simt(pl, k_pool, v_pool, q, out, lse, st));
+    }
+    return TESSERA_OK;
+}
+
+}  // namespace
+
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+}  // namespace tessera
+
+using namespace tessera;
+
+extern "C" {
+
+int32_t tessera_plan_create(const tessera_model_cfg *cfg, const tessera_compose_desc *desc, int32_t num_pool_pages,
+                            uint32_t flags, tessera_plan **out, void *stream) {
+    if (!out) return set_error(TESSERA_INVALID_ARG, "null out pointer");
+    *out = nullptr;
+    if (flags & ~uint32_t(TESSERA_PLAN_HOST_ONLY)) return set_error(TESSERA_INVALID_ARG, "unknown plan flag");
+    tessera_plan *pl = new (std::nothrow) tessera_plan();
+    if (!pl) return set_error(TESSERA_INVALID_ARG, "out of host memory");
+    std::string err;
+    int32_t st = TESSERA_INVALID_ARG;
+    try {
+        st = build_plan_host(cfg, desc, num_pool_pages, pl, &err);
+    } catch (const std::bad_alloc &) {
+        err = "out of host memory while building the plan";
+    }
+    if (st != TESSERA_OK) {
+        delete pl;
+        return set_error(st, err);
+    }
+    pl->host_only = (flags & TESSERA_PLAN_HOST_ONLY) != 0;
+    if (!pl->host_only) {
+        st = upload(pl, static_cast<cudaStream_t>(stream));
+        if (st != TESSERA_OK) {
+            if (pl->dev.blob) cudaFree(pl->dev.blob);
+            delete pl;
+            return st;
+        }
+    }
+    *out = pl;
+    return TESSERA_OK;
+}
+
+int32_t tessera_plan_destroy(tessera_plan *pl) {
+    if (!pl) return TESSERA_OK;
+    int32_t rc = TESSERA_OK;
+    if (!pl->host_only) {
+        void *bufs[] = {pl->dev.blob, pl->dev.st_q, pl->dev.st_k, pl->dev.st_v, pl->dev.st_o, pl->dev.st_lse};
+        for (void *b : bufs)
+            if (b) {
+                cudaError_t e = cudaFree(b);
+                if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree");
+            }
+    }
+    delete pl;
+    return rc;
+}
+
+int32_t tessera_plan_block_table(const tessera_plan *pl, const int32_t **page_off, const int32_t **pages,
+                                 const int32_t **src_slot) {
+    if (!pl) return set_error(TESSERA_INVALID_ARG, "null plan");
+    if (page_off) *page_off = pl->page_off.data();
+    if (pages) *pages = pl->pages.data();
+    if (src_slot) *src_slot = pl->src_slot.data();
+    return TESSERA_OK;
+}
+
+int32_t tessera_plan_get_info(const tessera_plan *pl, tessera_plan_info *info) {
+    if (!pl || !info) return set_error(TESSERA_INVALID_ARG, "null plan or info");
+    info->total_tokens = pl->total_tokens;
+    info->n_q = pl->n_q;
+    info->cached_tokens = pl->cached_tokens;
+    info->qk_pairs = pl->qk_pairs;
+    info->gather_bytes = pl->cached_tokens * pl->cfg.num_kv_heads * pl->cfg.head_dim * 2 * 2 * 2;
+    info->attn_flops = 4LL * pl->cfg.head_dim * pl->cfg.num_q_heads * pl->qk_pairs;
+    info->n_rope_rows = (int32_t)pl->rope_delta.size();
+    info->n_gather_items = (int32_t)pl->items.size();
+    info->n_attn_items = (int32_t)pl->tile_order.size();
+    info->attn_kernel = pl->attn_kernel;
+    return TESSERA_OK;
+}
+
+int32_t tessera_plan_status(tessera_plan *pl, int32_t *detail, void *stream) {
+    if (int32_t rc = check_device_plan(pl)) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t word[4] = {0, 0, 0, 0};
+    TS_CUDA(cudaMemcpyAsync(word, pl->dev.status, sizeof word, cudaMemcpyDeviceToHost, st));
+    TS_CUDA(cudaStreamSynchronize(st));
+    if (word[0] != 0) TS_CUDA(cudaMemsetAsync(pl->dev.status, 0, sizeof word, st));
+    if (detail) *detail = word[0];
+    if (word[0] != 0)
+        return set_error(TESSERA_DEVICE_TIMEOUT, "a bounded wait inside a kernel gave up, code " + std::to_string(word[0]));
+    return TESSERA_OK;
+}
+
+int32_t tessera_kv_compose(const tessera_plan *pl, void *k_pool, void *v_pool, uint32_t flags, void *stream) {
+    if (int32_t rc = check_device_plan(pl)) return rc;
+    if (flags & ~uint32_t(TESSERA_FUSE_ROPE)) return set_error(TESSERA_INVALID_ARG, "unknown compose flag");
+    if (!k_pool || !v_pool || misaligned(k_pool) || misaligned(v_pool))
+        return set_error(TESSERA_INVALID_ARG, "k_pool / v_pool must be non-null and 16-byte aligned");
+    TS_CUDA(launch_gather(pl, k_pool, v_pool, (flags & TESSERA_FUSE_ROPE) ? GatherMode::kCopyRotate : GatherMode::kCopy,
+                          static_cast<cudaStream_t>(stream)));
+    return TESSERA_OK;
+}
+
+int32_t tessera_rope_shift(const tessera_plan *pl, void *k_pool, void *stream) {
+    if (int32_t rc = check_device_plan(pl)) return rc;
+    if (!k_pool || misaligned(k_pool)) return set_error(TESSERA_INVALID_ARG, "k_pool must be non-null and 16-byte aligned");
+    TS_CUDA(launch_gather(pl, k_pool, k_pool, GatherMode::kShiftInPlace, static_cast<cudaStream_t>(stream)));
+    return TESSERA_OK;
+}
+
+int32_t tessera_partial_prefill_attn(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q,
+                                     const void *k_new, const void *v_new, void *out, float *lse, void *stream) {
+    if (int32_t rc = check_device_plan(pl)) return rc;
+    if (!k_pool || !v_pool || misaligned(k_pool) || misaligned(v_pool))
+        return set_error(TESSERA_INVALID_ARG, "k_pool / v_pool must be non-null and 16-byte aligned");
+    if (pl->n_q > 0 && (!q || !out)) return set_error(TESSERA_INVALID_ARG, "q and out must be non-null");
+    if (misaligned(q) || misaligned(out) || misaligned(k_new) || misaligned(v_new))
+        return set_error(TESSERA_INVALID_ARG, "q / out / k_new / v_new must be 16-byte aligned");
+    return attention(pl, k_pool, v_pool, q, k_new, v_new, out, lse, static_cast<cudaStream_t>(stream));
+}
+
+int32_t tessera_composed_prefill_host(tessera_plan *pl, void *k_pool, void *v_pool, const void *q_host,
+                                      const void *k_new_host, const void *v_new_host, void *out_host,
+                                      float *lse_host, void *stream) {
+    if (int32_t rc = check_device_plan(pl)) return rc;
+    if (!k_pool || !v_pool || misaligned(k_pool) || misaligned(v_pool))
+        return set_error(TESSERA_INVALID_ARG, "k_pool / v_pool must be non-null and 16-byte aligned");
+    if (pl->n_q > 0 && (!q_host || !k_new_host || !v_new_host || !out_host))
+        return set_error(TESSERA_INVALID_ARG, "q / k_new / v_new / out host buffers must be non-null");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DeviceTables &d = pl->dev;
+    const size_t q_bytes = (size_t)pl->n_q * pl->cfg.num_q_heads * pl->cfg.head_dim * 2;
+    const size_t kv_bytes = (size_t)pl->n_q * pl->cfg.num_kv_heads * pl->cfg.head_dim * 2;
+    const size_t lse_bytes = (size_t)pl->n_q * pl->cfg.num_q_heads * sizeof(float);
+    if (!d.st_q && pl->n_q > 0) {
+        TS_CUDA(cudaMalloc(&d.st_q, q_bytes));
+        TS_CUDA(cudaMalloc(&d.st_k, kv_bytes));
+        TS_CUDA(cudaMalloc(&d.st_v, kv_bytes));
+        TS_CUDA(cudaMalloc(&d.st_o, q_bytes));
+        TS_CUDA(cudaMalloc(reinterpret_cast<void **>(&d.st_lse), lse_bytes));
+    }
+    if (pl->n_q > 0) {
+        TS_CUDA(cudaMemcpyAsync(d.st_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
+        TS_CUDA(cudaMemcpyAsync(d.st_k, k_new_host, kv_bytes, cudaMemcpyHostToDevice, st));
+        TS_CUDA(cudaMemcpyAsync(d.st_v, v_new_host, kv_bytes, cudaMemcpyHostToDevice, st));
+    }
+    TS_CUDA(launch_gather(pl, k_pool, v_pool, GatherMode::kCopyRotate, st));
+    if (int32_t rc = attention(pl, k_pool, v_pool, d.st_q, d.st_k, d.st_v, d.st_o, d.st_lse, st)) return rc;
+    if (pl->n_q > 0) {
+        TS_CUDA(cudaMemcpyAsync(out_host, d.st_o, q_bytes, cudaMemcpyDeviceToHost, st));
+        if (lse_host) TS_CUDA(cudaMemcpyAsync(lse_host, d.st_lse, lse_bytes, cudaMemcpyDeviceToHost, st));
+    }
+    TS_CUDA(cudaStreamSynchronize(st));
+    return TESSERA_OK;
+}
+
+int32_t tessera_last_error(char *buf, int32_t len) {
+    const std::string &e = g_last_error;
+    if (buf && len > 0) {
+        const size_t n = std::min<size_t>(e.size(), (size_t)len - 1);
+        std::memcpy(buf, e.data(), n);
+        buf[n] = 0;
+    }
+    return (int32_t)e.size();
+}
+
+int64_t tessera_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,198 @@
+// Gather + RoPE shift (HBM-bound) and the fresh-row scatter.
+//
+// gather_rope_kernel moves cached token rows from their source slots to the request's destination
+// slots (Sec. 5.3 "Preparing cache hits").  V rows are bit copies; K rows are either bit copies or
+// rotated by the unit's shift on the way (Sec. 2.2: keys carry the rotation, values do not).
+// Every global access is a 16-byte chunk; the two halves of a rotary pair (m, m + D/2) of one head
+// are loaded by the same thread, so no data crosses lanes.  The cos/sin rows an item needs are
+// staged in shared memory once per thread block.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "launch.h"
+#include "plan.h"
+
+namespace tessera {
+
+namespace {
+
+__device__ __forceinline__ uint4 ldg_stream(const uint4 *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint4 ldg_plain(const uint4 *p) {
+    uint4 v;
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void stg(uint4 *p, const uint4 &v) {
+    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// Rotates 8 pairs: lo holds x_m, hi holds x_{m + D/2}, cs[i] = (cos, sin) of pair i.
+// x' = x cos - y sin, y' = y cos + x sin in fp32, one round-to-nearest-even to bf16.
+__device__ __forceinline__ void rotate8(uint4 &lo, uint4 &hi, const float2 *cs) {
+    uint32_t *l = reinterpret_cast<uint32_t *>(&lo);
+    uint32_t *h = reinterpret_cast<uint32_t *>(&hi);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float x0 = __uint_as_float(l[i] << 16), x1 = __uint_as_float(l[i] & 0xffff0000u);
+        const float y0 = __uint_as_float(h[i] << 16), y1 = __uint_as_float(h[i] & 0xffff0000u);
+        const float2 c0 = cs[2 * i], c1 = cs[2 * i + 1];
+        const float a0 = fmaf(-y0, c0.y, x0 * c0.x), a1 = fmaf(-y1, c1.y, x1 * c1.x);
+        const float b0 = fmaf(x0, c0.y, y0 * c0.x), b1 = fmaf(x1, c1.y, y1 * c1.x);
+        __nv_bfloat162 pa = __floats2bfloat162_rn(a0, a1), pb = __floats2bfloat162_rn(b0, b1);
+        l[i] = *reinterpret_cast<uint32_t *>(&pa);
+        h[i] = *reinterpret_cast<uint32_t *>(&pb);
+    }
+}
+
+constexpr int kThreads = 256;
+
+// One thread block per GatherItem.  A "task" is one rotary pair-chunk of one token row: the 16-byte
+// chunk holding elements [8c, 8c+8) of a head and its partner chunk D/2 elements later (K), plus the
+// same two chunks of the V row.  IN_PLACE: source = destination, K only (the standalone shift).
+template <int D, bool DO_V, bool ROTATE, bool IN_PLACE>
+__global__ void __launch_bounds__(kThreads)
+gather_rope_kernel(uint4 *__restrict__ k_pool, uint4 *__restrict__ v_pool,
+                   const int32_t *__restrict__ g_src, const int32_t *__restrict__ g_dst,
+                   const GatherItem *__restrict__ items, const float2 *__restrict__ rope, int H_kv) {
+    constexpr int CPH = D / 16;          // pair-chunks per head
+    constexpr int HALF = D / 16;         // distance (in 16-byte chunks) between pair partners
+    __shared__ float2 s_rope[kGatherItemTokens * (D / 2)];
+    __shared__ int32_t s_src[kGatherItemTokens], s_dst[kGatherItemTokens];
+
+    const GatherItem it = items[blockIdx.x];
+    const int tid = threadIdx.x;
+    const int n_rows = ROTATE ? (it.row_step ? it.count : 1) : 0;
+    for (int i = tid; i < n_rows * (D / 2); i += kThreads) s_rope[i] = rope[(size_t)it.row0 * (D / 2) + i];
+    if (tid < it.count) {
+        s_dst[tid] = g_dst[it.begin + tid];
+        s_src[tid] = IN_PLACE ? s_dst[tid] : g_src[it.begin + tid];
+    }
+    __syncthreads();
+
+    const int tasks_per_row = H_kv * CPH;
+    const int row_chunks = H_kv * (D / 8);
+    const int n_tasks = it.count * tasks_per_row;
+    const int c = tid % CPH;             // kThreads and tasks_per_row are multiples of CPH
+    float2 cs[8];
+    if (ROTATE && it.row_step == 0) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cs[i] = s_rope[c * 8 + i];
+    }
+
+    constexpr int U = 2;                 // tasks in flight per thread
+    for (int t0 = tid; t0 < n_tasks; t0 += U * kThreads) {
+        uint4 klo[U], khi[U], vlo[U], vhi[U];
+        size_t dsto[U];
+        int tok[U];
+        bool ok[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int t = t0 + u * kThreads;
+            ok[u] = t < n_tasks;
+            if (!ok[u]) continue;
+            tok[u] = t / tasks_per_row;
+            const int w = t - tok[u] * tasks_per_row;
+            const int chunk = (w / CPH) * (D / 8) + c;
+            const size_t so = (size_t)s_src[tok[u]] * row_chunks + chunk;
+            dsto[u] = (size_t)s_dst[tok[u]] * row_chunks + chunk;
+            if (IN_PLACE) {
+                klo[u] = ldg_plain(k_pool + so);
+                khi[u] = ldg_plain(k_pool + so + HALF);
+            } else {
+                klo[u] = ldg_stream(k_pool + so);
+                khi[u] = ldg_stream(k_pool + so + HALF);
+            }
+            if (DO_V) {
+                vlo[u] = ldg_stream(v_pool + so);
+                vhi[u] = ldg_stream(v_pool + so + HALF);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (!ok[u]) continue;
+            if (DO_V) {
+                stg(v_pool + dsto[u], vlo[u]);
+                stg(v_pool + dsto[u] + HALF, vhi[u]);
+            }
+            if (ROTATE) {
+                if (it.row_step != 0) {
+                    const float2 *row = s_rope + (size_t)tok[u] * (D / 2) + c * 8;
+                    float2 cr[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) cr[i] = row[i];
+                    rotate8(klo[u], khi[u], cr);
+                } else {
+                    rotate8(klo[u], khi[u], cs);
+                }
+            }
+            stg(k_pool + dsto[u], klo[u]);
+            stg(k_pool + dsto[u] + HALF, khi[u]);
+        }
+    }
+}
+
+// Writes the recomputed K / V rows into their destination slots (Sec. 5.3 "Completing prefill":
+// recomputed states are private to the request and override the cached ones).
+__global__ void __launch_bounds__(256)
+scatter_fresh_kernel(uint4 *__restrict__ k_pool, uint4 *__restrict__ v_pool,
+                     const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
+                     const int32_t *__restrict__ fresh_dst, int64_t n_chunks, int row_chunks) {
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_chunks; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t j = e / row_chunks;
+        const int c = (int)(e - j * row_chunks);
+        const size_t o = (size_t)fresh_dst[j] * row_chunks + c;
+        if (k_new) stg(k_pool + o, ldg_stream(k_new + e));
+        if (v_new) stg(v_pool + o, ldg_stream(v_new + e));
+    }
+}
+
+template <int D>
+cudaError_t launch_gather_d(const tessera_plan *pl, void *k_pool, void *v_pool, GatherMode mode, cudaStream_t st) {
+    const int n = (int)pl->items.size();
+    if (n == 0) return cudaSuccess;
+    auto *kp = static_cast<uint4 *>(k_pool);
+    auto *vp = static_cast<uint4 *>(v_pool);
+    const DeviceTables &d = pl->dev;
+    const int H = pl->cfg.num_kv_heads;
+    switch (mode) {
+        case GatherMode::kCopy:
+            gather_rope_kernel<D, true, false, false><<<n, kThreads, 0, st>>>(kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            break;
+        case GatherMode::kCopyRotate:
+            gather_rope_kernel<D, true, true, false><<<n, kThreads, 0, st>>>(kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            break;
+        case GatherMode::kShiftInPlace:
+            gather_rope_kernel<D, false, true, true><<<n, kThreads, 0, st>>>(kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            break;
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_gather(const tessera_plan *pl, void *k_pool, void *v_pool, GatherMode mode, cudaStream_t st) {
+    return pl->cfg.head_dim == 128 ? launch_gather_d<128>(pl, k_pool, v_pool, mode, st)
+                                   : launch_gather_d<64>(pl, k_pool, v_pool, mode, st);
+}
+
+cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_pool, const void *k_new,
+                                 const void *v_new, cudaStream_t st) {
+    if (pl->n_q == 0 || (!k_new && !v_new)) return cudaSuccess;
+    const int row_chunks = pl->cfg.num_kv_heads * pl->cfg.head_dim / 8;
+    const int64_t n_chunks = pl->n_q * row_chunks;
+    const int blocks = (int)std::min<int64_t>((n_chunks + 255) / 256, 148 * 16);
+    scatter_fresh_kernel<<<blocks, 256, 0, st>>>(static_cast<uint4 *>(k_pool), static_cast<uint4 *>(v_pool),
+                                                static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new),
+                                                pl->dev.fresh_dst, n_chunks, row_chunks);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace tessera

@@ -1,0 +1,22 @@
+// Launch entry points of the individual kernels (internal to the library).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "plan.h"
+
+namespace tessera {
+
+enum class GatherMode { kCopy, kCopyRotate, kShiftInPlace };
+
+void count_launch();   // bumps the process-wide kernel-launch counter
+
+cudaError_t launch_gather(const tessera_plan *pl, void *k_pool, void *v_pool, GatherMode mode, cudaStream_t st);
+cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_pool, const void *k_new,
+                                 const void *v_new, cudaStream_t st);
+cudaError_t launch_attn_simt(const tessera_plan *pl, const void *k_pool, const void *v_pool, const void *q,
+                             void *out, float *lse, cudaStream_t st);
+// tcgen05 path; returns cudaErrorNotSupported when the plan's shape is outside its range.
+cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
+                           float *lse, cudaStream_t st, std::string *err);
+
+}  // namespace tessera

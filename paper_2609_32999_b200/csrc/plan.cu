@@ -1,0 +1,232 @@
+// Host-side placement: validation of a batch descriptor and construction of every table the
+// kernels read (Sec. 5.3 "Placement before preparation"; storage blocks of Sec. 5.1).
+// Pure host code: it makes no CUDA call, so it also runs where no GPU exists.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <numeric>
+
+#include <vector_types.h>
+
+#include "plan.h"
+
+namespace tessera {
+
+namespace {
+
+std::string fmt(const char *f, long a = 0, long b = 0, long c = 0) {
+    char buf[256];
+    snprintf(buf, sizeof buf, f, a, b, c);
+    return buf;
+}
+
+bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+
+}  // namespace
+
+int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc *d,
+                        int32_t num_pool_pages, tessera_plan *pl, std::string *err) {
+    auto fail = [&](int32_t code, const std::string &msg) { *err = msg; return code; };
+    if (!cfg || !d || !pl) return fail(TESSERA_INVALID_ARG, "null cfg / desc / plan");
+    if (d->batch < 0 || num_pool_pages < 0 || d->n_free < 0)
+        return fail(TESSERA_INVALID_ARG, "negative batch, pool size or free-list length");
+    if (d->batch > 0 && (!d->seq_len || !d->unit_off || !d->recompute_off))
+        return fail(TESSERA_INVALID_ARG, "null seq_len / unit_off / recompute_off");
+
+    // ---- shapes the kernels cover
+    const int Hq = cfg->num_q_heads, Hkv = cfg->num_kv_heads, D = cfg->head_dim, B = cfg->page_size;
+    if (Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0)
+        return fail(TESSERA_UNSUPPORTED_SHAPE, fmt("num_q_heads %ld must be a positive multiple of num_kv_heads %ld", Hq, Hkv));
+    if (Hq / Hkv > 16) return fail(TESSERA_UNSUPPORTED_SHAPE, "group size H_q/H_kv above 16");
+    if (D != 64 && D != 128) return fail(TESSERA_UNSUPPORTED_SHAPE, fmt("head_dim %ld: only 64 and 128", D));
+    if (B <= 0 || B % 8 != 0 || B > 128 || !is_pow2(B))
+        return fail(TESSERA_UNSUPPORTED_SHAPE, fmt("page_size %ld: a power of two in 8..128", B));
+    if (cfg->rope_pairing != 0) return fail(TESSERA_UNSUPPORTED_SHAPE, "rope_pairing: only 0 (half-split pairs)");
+    if (!cfg->inv_freq && !(cfg->rope_theta > 0.0)) return fail(TESSERA_INVALID_ARG, "rope_theta must be positive");
+    if ((int64_t)num_pool_pages * B > (int64_t)INT32_MAX)
+        return fail(TESSERA_UNSUPPORTED_SHAPE, "pool has more than 2^31 slots");
+
+    pl->cfg = *cfg;
+    pl->inv_freq.resize(D / 2);
+    for (int m = 0; m < D / 2; ++m)
+        pl->inv_freq[m] = cfg->inv_freq ? cfg->inv_freq[m] : std::pow(cfg->rope_theta, -2.0 * m / D);
+    pl->cfg.inv_freq = nullptr;
+    pl->sm_scale = cfg->sm_scale != 0.f ? cfg->sm_scale : (float)(1.0 / std::sqrt((double)D));
+    pl->num_pool_pages = num_pool_pages;
+    pl->batch = d->batch;
+
+    const int batch = d->batch;
+    // ---- CSR sanity
+    if (batch > 0) {
+        if (d->unit_off[0] != 0 || d->recompute_off[0] != 0) return fail(TESSERA_INVALID_ARG, "CSR offsets must start at 0");
+        for (int r = 0; r < batch; ++r) {
+            if (d->seq_len[r] < 0) return fail(TESSERA_INVALID_ARG, fmt("request %ld: negative seq_len", r));
+            if (d->unit_off[r + 1] < d->unit_off[r] || d->recompute_off[r + 1] < d->recompute_off[r])
+                return fail(TESSERA_INVALID_ARG, fmt("request %ld: CSR offsets decrease", r));
+        }
+    }
+    const int n_units = batch ? d->unit_off[batch] : 0;
+    const int n_q = batch ? d->recompute_off[batch] : 0;
+    if (n_units > 0 && (!d->unit_len || !d->unit_cached_pos || !d->unit_cached_stride || !d->unit_target_pos || !d->unit_page_off))
+        return fail(TESSERA_INVALID_ARG, "null unit array");
+    if (n_q > 0 && !d->recompute_pos) return fail(TESSERA_INVALID_ARG, "null recompute_pos");
+    if (n_units > 0) {
+        if (d->unit_page_off[0] != 0) return fail(TESSERA_INVALID_ARG, "unit_page_off must start at 0");
+        for (int u = 0; u < n_units; ++u) {
+            if (d->unit_len[u] < 0) return fail(TESSERA_INVALID_ARG, fmt("unit %ld: negative length", u));
+            int np = d->unit_page_off[u + 1] - d->unit_page_off[u];
+            if (np < 0) return fail(TESSERA_INVALID_ARG, fmt("unit %ld: unit_page_off decreases", u));
+            if (np != 0 && np != (d->unit_len[u] + B - 1) / B)
+                return fail(TESSERA_INVALID_ARG, fmt("unit %ld: %ld source pages for %ld tokens", u, np, d->unit_len[u]));
+            if (np != 0 && d->unit_cached_stride[u] != 0 && d->unit_cached_stride[u] != 1)
+                return fail(TESSERA_INVALID_ARG, fmt("unit %ld: cached stride must be 0 or 1", u));
+        }
+        if (d->unit_page_off[n_units] > 0 && !d->unit_pages) return fail(TESSERA_INVALID_ARG, "null unit_pages");
+    }
+
+    // ---- block tables: request r takes the next ceil(T_r / B) free pages
+    pl->seq_len.assign(d->seq_len, d->seq_len + batch);
+    pl->tok_off.assign(batch + 1, 0);
+    pl->page_off.assign(batch + 1, 0);
+    int64_t total = 0, need_pages = 0;
+    for (int r = 0; r < batch; ++r) {
+        total += d->seq_len[r];
+        need_pages += (d->seq_len[r] + B - 1) / B;
+        if (total > INT32_MAX) return fail(TESSERA_UNSUPPORTED_SHAPE, "batch has more than 2^31 tokens");
+        pl->tok_off[r + 1] = (int32_t)total;
+        pl->page_off[r + 1] = (int32_t)need_pages;
+    }
+    if (need_pages > d->n_free)
+        return fail(TESSERA_OUT_OF_PAGES, fmt("batch needs %ld destination pages, free list has %ld", need_pages, d->n_free));
+    if (need_pages > 0 && !d->free_pages) return fail(TESSERA_INVALID_ARG, "null free_pages");
+    pl->pages.assign(d->free_pages, d->free_pages + need_pages);
+
+    // page ids: range, destinations distinct, destinations disjoint from sources
+    std::vector<uint8_t> page_use(num_pool_pages, 0);   // 1 = source, 2 = destination
+    const int n_src_pages = n_units ? d->unit_page_off[n_units] : 0;
+    for (int k = 0; k < n_src_pages; ++k) {
+        int pg = d->unit_pages[k];
+        if (pg < 0 || pg >= num_pool_pages) return fail(TESSERA_PAGE_OUT_OF_RANGE, fmt("source page %ld outside pool of %ld pages", pg, num_pool_pages));
+        page_use[pg] = 1;
+    }
+    for (int64_t k = 0; k < need_pages; ++k) {
+        int pg = pl->pages[k];
+        if (pg < 0 || pg >= num_pool_pages) return fail(TESSERA_PAGE_OUT_OF_RANGE, fmt("free page %ld outside pool of %ld pages", pg, num_pool_pages));
+        if (page_use[pg] == 1) return fail(TESSERA_PAGE_OUT_OF_RANGE, fmt("free page %ld is also a source page of this batch", pg));
+        if (page_use[pg] == 2) return fail(TESSERA_PAGE_OUT_OF_RANGE, fmt("free page %ld listed twice", pg));
+        page_use[pg] = 2;
+    }
+
+    // ---- per-position sources, recompute rows, coverage
+    pl->src_slot.assign((size_t)total, -1);
+    pl->recompute_off.assign(d->recompute_off, d->recompute_off + batch + 1);
+    pl->recompute_pos.assign(d->recompute_pos, d->recompute_pos + n_q);
+    pl->q_req.resize(n_q);
+    pl->fresh_dst.resize(n_q);
+    pl->g_src.clear(); pl->g_dst.clear(); pl->items.clear();
+    std::vector<int32_t> unit_of((size_t)total, -1);
+    std::vector<uint8_t> fresh((size_t)total, 0);
+    std::vector<int64_t> deltas;     // shift amounts needed, with repeats
+    pl->qk_pairs = 0;
+    for (int r = 0; r < batch; ++r) {
+        const int T = d->seq_len[r];
+        const int64_t base = pl->tok_off[r];
+        for (int u = d->unit_off[r]; u < d->unit_off[r + 1]; ++u) {
+            const int len = d->unit_len[u], tp = d->unit_target_pos[u];
+            if (tp < 0 || (int64_t)tp + len > T)
+                return fail(TESSERA_UNIT_OVERLAP, fmt("unit %ld leaves its request's positions [0, %ld)", u, T));
+            const bool cached = d->unit_page_off[u + 1] > d->unit_page_off[u];
+            for (int i = 0; i < len; ++i) {
+                if (unit_of[base + tp + i] != -1)
+                    return fail(TESSERA_UNIT_OVERLAP, fmt("units %ld and %ld both claim position %ld", unit_of[base + tp + i], u, tp + i));
+                unit_of[base + tp + i] = u;
+                if (cached)
+                    pl->src_slot[base + tp + i] = d->unit_pages[d->unit_page_off[u] + i / B] * B + i % B;
+            }
+        }
+        for (int j = d->recompute_off[r]; j < d->recompute_off[r + 1]; ++j) {
+            const int p = d->recompute_pos[j];
+            if (p < 0 || p >= T) return fail(TESSERA_INVALID_ARG, fmt("request %ld: recompute position %ld outside [0, %ld)", r, p, T));
+            if (j > d->recompute_off[r] && d->recompute_pos[j - 1] >= p)
+                return fail(TESSERA_UNSORTED_POSITIONS, fmt("request %ld: recompute positions not strictly ascending at index %ld", r, j));
+            fresh[base + p] = 1;
+            pl->q_req[j] = r;
+            pl->fresh_dst[j] = pl->pages[pl->page_off[r] + p / B] * B + p % B;
+            pl->qk_pairs += (int64_t)p + 1;
+        }
+        for (int p = 0; p < T; ++p)
+            if (pl->src_slot[base + p] < 0 && !fresh[base + p])
+                return fail(TESSERA_UNCOVERED_POSITION, fmt("request %ld: position %ld has no cached unit and is not recomputed", r, p));
+    }
+
+    // ---- copy list + shift table.  One item = up to kGatherItemTokens rows of one unit.
+    for (int r = 0; r < batch; ++r)
+        for (int u = d->unit_off[r]; u < d->unit_off[r + 1]; ++u) {
+            if (d->unit_page_off[u + 1] <= d->unit_page_off[u]) continue;
+            const int64_t d0 = (int64_t)d->unit_target_pos[u] - d->unit_cached_pos[u];
+            if (d->unit_cached_stride[u] == 1) deltas.push_back(d0);
+            else for (int i = 0; i < d->unit_len[u]; ++i) deltas.push_back(d0 + i);
+        }
+    std::sort(deltas.begin(), deltas.end());
+    deltas.erase(std::unique(deltas.begin(), deltas.end()), deltas.end());
+    for (int64_t x : deltas)
+        if (x > INT32_MAX || x < INT32_MIN) return fail(TESSERA_INVALID_ARG, "shift amount overflows int32");
+    pl->rope_delta.assign(deltas.begin(), deltas.end());
+    pl->rope_table.resize(deltas.size() * (size_t)D);     // [row][D/2][cos, sin]
+    for (size_t row = 0; row < deltas.size(); ++row)
+        for (int m = 0; m < D / 2; ++m) {
+            // angle, cosine and sine in fp64; a single rounding to fp32 each
+            const double ang = (double)deltas[row] * pl->inv_freq[m];
+            pl->rope_table[(row * (D / 2) + m) * 2 + 0] = (float)std::cos(ang);
+            pl->rope_table[(row * (D / 2) + m) * 2 + 1] = (float)std::sin(ang);
+        }
+    auto row_of = [&](int64_t delta) {
+        return (int32_t)(std::lower_bound(deltas.begin(), deltas.end(), delta) - deltas.begin());
+    };
+    pl->cached_tokens = 0;
+    for (int r = 0; r < batch; ++r)
+        for (int u = d->unit_off[r]; u < d->unit_off[r + 1]; ++u) {
+            if (d->unit_page_off[u + 1] <= d->unit_page_off[u]) continue;
+            const int len = d->unit_len[u], tp = d->unit_target_pos[u];
+            const int64_t d0 = (int64_t)tp - d->unit_cached_pos[u];
+            const int step = d->unit_cached_stride[u] == 1 ? 0 : 1;
+            const int32_t row0 = row_of(d0);       // stride 0: consecutive integers are consecutive rows
+            for (int i0 = 0; i0 < len; i0 += kGatherItemTokens) {
+                const int cnt = std::min(kGatherItemTokens, len - i0);
+                pl->items.push_back({(int32_t)pl->g_src.size(), cnt, row0 + i0 * step, step});
+                for (int i = i0; i < i0 + cnt; ++i) {
+                    const int p = tp + i;
+                    pl->g_src.push_back(pl->src_slot[pl->tok_off[r] + p]);
+                    pl->g_dst.push_back(pl->pages[pl->page_off[r] + p / B] * B + p % B);
+                }
+            }
+            pl->cached_tokens += len;
+        }
+
+    // ---- attention work list: tiles of consecutive recompute rows of one request
+    const int g = Hq / Hkv;
+    pl->attn_kernel = 0;
+    pl->tile_tokens = kAttnTileRows / g;
+    if (kHaveTensorCoreKernel && D == 128 && B == 64 && kAttnTileRows % g == 0) pl->attn_kernel = 1;
+    pl->tiles.clear();
+    for (int r = 0; r < batch; ++r)
+        for (int j0 = d->recompute_off[r]; j0 < d->recompute_off[r + 1]; j0 += pl->tile_tokens) {
+            const int n = std::min(pl->tile_tokens, d->recompute_off[r + 1] - j0);
+            AttnTile t{};
+            t.req = r; t.q_begin = j0; t.n_tok = n;
+            t.kv_len = d->recompute_pos[j0 + n - 1] + 1;
+            t.kv_full = d->recompute_pos[j0] + 1;
+            pl->tiles.push_back(t);
+        }
+    pl->tile_order.resize(pl->tiles.size() * (size_t)Hkv);
+    std::iota(pl->tile_order.begin(), pl->tile_order.end(), 0);
+    std::stable_sort(pl->tile_order.begin(), pl->tile_order.end(), [&](int32_t a, int32_t b) {
+        return pl->tiles[a / Hkv].kv_len > pl->tiles[b / Hkv].kv_len;
+    });
+
+    pl->total_tokens = total;
+    pl->n_q = n_q;
+    return TESSERA_OK;
+}
+
+}  // namespace tessera

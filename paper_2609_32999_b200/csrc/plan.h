@@ -1,0 +1,79 @@
+// Internal plan representation shared by the host builder and the launch code.
+#pragma once
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include <vector_types.h>
+
+#include "tessera.h"
+
+namespace tessera {
+
+constexpr int kGatherItemTokens = 32;   // token rows per thread block of the gather kernel
+constexpr int kAttnTileRows = 128;      // query rows (tokens x grouped heads) per tcgen05 tile
+constexpr bool kHaveTensorCoreKernel = false;
+
+// One thread block of the gather / shift kernel: `count` consecutive entries of the copy list that
+// belong to one cached unit.  Entry i uses row (row0 + i * row_step) of the cos/sin table.
+struct GatherItem {
+    int32_t begin, count, row0, row_step;
+};
+
+// One query tile of the attention kernel: `n_tok` consecutive recompute rows [q_begin, q_begin+n_tok)
+// of request `req`; the tile reads keys [0, kv_len).  Keys below `kv_full` are visible to every row.
+struct AttnTile {
+    int32_t req, q_begin, n_tok, kv_len, kv_full, pad0, pad1, pad2;
+};
+
+struct DeviceTables {
+    void *blob = nullptr;          // one allocation holding everything below
+    int32_t *g_src = nullptr, *g_dst = nullptr;
+    GatherItem *items = nullptr;
+    float2 *rope = nullptr;        // [n_rope_rows][D/2] (cos, sin)
+    int32_t *fresh_dst = nullptr;  // [n_q] destination slot of each recompute row
+    int32_t *q_pos = nullptr;      // [n_q]
+    int32_t *q_req = nullptr;      // [n_q]
+    int32_t *page_off = nullptr;   // [batch+1]
+    int32_t *pages = nullptr;      // block tables
+    AttnTile *tiles = nullptr;
+    int32_t *tile_order = nullptr; // work items (tile * H_kv + kv head), longest first
+    int32_t *status = nullptr;     // device status word(s)
+    // staging for the host-buffer entry point (allocated on first use)
+    void *st_q = nullptr, *st_k = nullptr, *st_v = nullptr, *st_o = nullptr;
+    float *st_lse = nullptr;
+};
+
+}  // namespace tessera
+
+struct tessera_plan {
+    tessera_model_cfg cfg{};
+    std::vector<double> inv_freq;          // [D/2], always filled
+    float sm_scale = 0.f;
+    int32_t num_pool_pages = 0;
+    int32_t batch = 0;
+    bool host_only = false;
+    int device = -1;
+
+    std::vector<int32_t> seq_len, tok_off, page_off, pages, src_slot;
+    std::vector<int32_t> recompute_off, recompute_pos, q_req, fresh_dst;
+    std::vector<int32_t> g_src, g_dst;
+    std::vector<tessera::GatherItem> items;
+    std::vector<int32_t> rope_delta;       // sorted distinct shift amounts
+    std::vector<float> rope_table;         // [rows][D/2][2]
+    std::vector<tessera::AttnTile> tiles;
+    std::vector<int32_t> tile_order;
+    int32_t attn_kernel = 0;
+    int32_t tile_tokens = 0;
+
+    int64_t total_tokens = 0, n_q = 0, cached_tokens = 0, qk_pairs = 0;
+
+    std::vector<char> host_blob;           // staging image of the device tables
+    tessera::DeviceTables dev;
+};
+
+namespace tessera {
+// Builds and validates all host tables.  Returns a status; on failure `err` holds the reason.
+int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc *desc,
+                        int32_t num_pool_pages, tessera_plan *plan, std::string *err);
+}  // namespace tessera

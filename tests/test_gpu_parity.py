@@ -1,0 +1,154 @@
+"""GPU parity: the CUDA library against the fp64 oracle on the same seeded bytes, through the C ABI."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import tessera_oracle as orc
+from paper_2609_32999_b200 import binding as tb
+from paper_2609_32999_b200 import workloads as wl
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+def _full_check(w, fuse=True, seed=None):
+    g = gu.run_layer(w, fuse=fuse, seed=seed)
+    assert g.status == 0
+    gu.check_placement(g)
+    asm, kmx, kmean = gu.check_assembled(g)
+    gu.check_untouched(g)
+    amx, amean = gu.check_attention(g, asm)                       # whole path vs unrounded oracle keys
+    gu.check_attention(g, asm, use_pool_k=True)                   # attention kernel alone
+    return g, (kmx, kmean, amx, amean)
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3])
+def test_config_full_parity(idx):
+    _full_check(wl.config(idx))
+
+
+def test_adversarial_shapes_and_shifts():
+    """Negative shifts, non-zero cached positions, keys cached without rotation, a unit used twice,
+    ragged pages, an uncached unit, an empty-ish request; small head_dim path and the Llama shape."""
+    _full_check(wl.adversarial())
+    _full_check(wl.adversarial(seed=9, shape=wl.ModelShape(32, 8, 128, 64, 500000.0)))
+    _full_check(wl.adversarial(seed=10, shape=wl.ModelShape(16, 2, 128, 64, 500000.0)))
+    _full_check(wl.adversarial(seed=11, shape=wl.ModelShape(8, 8, 128, 64, 10000.0)))
+
+
+def test_unfused_compose_then_shift_equals_fused():
+    w = wl.config(3, requests_override=4)
+    a = gu.run_layer(w, fuse=True, seed=5, attention=False)
+    b = gu.run_layer(w, fuse=False, seed=5, attention=False)
+    assert np.array_equal(a.k_before, b.k_before)
+    assert np.array_equal(a.k_after, b.k_after) and np.array_equal(a.v_after, b.v_after)
+    gu.check_assembled(b, scattered=False)
+
+
+def test_zero_shift_is_bit_copy():
+    """A unit reused at the position it was cached at must come through bit for bit."""
+    shape = wl.ModelShape(32, 8, 128, 64, 500000.0)
+    segs = [wl.unit(300, "a", cached_pos=0, recompute=(0,)), wl.unit(200, "b", cached_pos=300, recompute=(0,)), 5]
+    w = wl.build_workload("zero", shape, [segs], np.random.default_rng(1))
+    g = gu.run_layer(w, attention=False)
+    asm, mx, mean = gu.check_assembled(g, scattered=False)
+    assert mx == 0.0 and np.all(asm[0].delta == 0)
+
+
+def test_uniform_softmax_lse_and_mean():
+    """K == 0: LSE = ln(p + 1) and O = mean of V[0..p] - shows the causal limit and page skipping
+    exactly, which the absolute tolerance alone cannot at long context."""
+    for w in (wl.config(1), wl.config(2), wl.adversarial(seed=9, shape=wl.ModelShape(32, 8, 128, 64, 500000.0))):
+        t = wl.make_tensors(w, device="cuda:0")
+        t.k_pool.zero_(); t.k_new.zero_()
+        D = w.shape.head_dim
+        sl = torch.arange(w.num_pool_pages * w.shape.page_size, device="cuda:0")
+        v = torch.nn.functional.one_hot(sl % D, D).to(torch.bfloat16)          # V[slot] = e_(slot mod D)
+        t.v_pool.copy_(v.view(w.num_pool_pages, w.shape.page_size, 1, D).expand_as(t.v_pool))
+        t.v_new.zero_()
+        g = gu.run_layer(w, t=t, poison=False)
+        assert g.status == 0
+        asm, _, _ = gu.check_assembled(g)
+        for r, a in asm.items():
+            jj, hh, pp = orc.request_rows(w, r)
+            if len(jj) == 0:
+                continue
+            assert np.max(np.abs(g.lse_f[jj, hh] - np.log(pp + 1.0))) < 2e-4
+            o, _ = orc.attention_rows(w, a.k, a.v_bits, g.q_bits, jj, hh, pp)
+            # outputs are counts / (p + 1): exact up to the final bf16 rounding (relative 2^-8)
+            assert np.all(np.abs(g.out_f[jj, hh] - o) <= np.abs(o) * 2.0 ** -8 + 1e-6)
+
+
+def test_needle_on_each_side_of_causal_limit_and_page_boundary():
+    shape = wl.ModelShape(32, 8, 128, 64, 500000.0)
+    T = 64 * 5
+    w = wl.build_workload("needle", shape, [[wl.unit(T, "a", cached=False)]], np.random.default_rng(3))
+    dev = "cuda:0"
+    for needle in (62, 63, 64, 65, 127, 128, 129, 255, 256, 257):
+        t = wl.make_tensors(w, device=dev)
+        t.q.zero_(); t.q[:, :, 0] = 8.0
+        t.k_new.zero_(); t.k_new[needle, :, 0] = 64.0
+        t.v_new.zero_(); t.v_new[needle, :, 1] = 1.0
+        g = gu.run_layer(w, t=t, poison=True)
+        col = g.out_f[:, :, 1]
+        assert np.all(col[:needle] == 0.0), needle
+        assert np.all(col[needle:] > 0.99), needle
+
+
+def test_deterministic_and_null_lse():
+    w = wl.config(3, requests_override=3)
+    a = gu.run_layer(w, seed=1)
+    b = gu.run_layer(w, seed=1, with_lse=False)
+    assert torch.equal(a.out, b.out)
+    assert np.array_equal(a.k_after, b.k_after)
+
+
+def test_explicit_inv_freq_overrides_theta():
+    w = wl.config(1)
+    D = w.shape.head_dim
+    inv = (w.shape.rope_theta ** (-2.0 * np.arange(D // 2) / D)) * 0.5       # scaled frequencies
+    plan = tb.Plan(w, inv_freq=inv)
+    g = gu.run_layer(w, plan=plan, attention=False)
+    sh = w.shape
+    row = sh.num_kv_heads * sh.head_dim
+    a = orc.assemble(w, 0, g.k_before, g.v_before, g.kn_bits, g.vn_bits, inv_freq=inv)
+    gk = orc.bf16_bits_to_f64(g.k_after.reshape(-1, row)[gu.dest_slots(g, 0)])
+    rot = a.k_exact == 0
+    rot[w.recompute_pos] = False
+    d = np.abs(gk[rot] - a.k.reshape(-1, row)[rot])
+    assert d.max() <= gu.MAX_ABS and d.mean() <= gu.MEAN_ABS
+    wrong = orc.assemble(w, 0, g.k_before, g.v_before, g.kn_bits, g.vn_bits)
+    assert np.abs(gk[rot] - wrong.k.reshape(-1, row)[rot]).max() > 0.5
+
+
+def test_host_buffer_entry_point_matches_device_calls():
+    w = wl.config(2)
+    g = gu.run_layer(w, seed=2)
+    t = wl.make_tensors(w, device="cuda:0", seed=2)
+    plan = tb.Plan(w)
+    qh, kh, vh = (x.cpu().pin_memory() for x in (t.q, t.k_new, t.v_new))
+    oh = torch.empty_like(qh).pin_memory()
+    lh = torch.empty(w.n_q, w.shape.num_q_heads, dtype=torch.float32).pin_memory()
+    plan.composed_prefill_host(t.k_pool, t.v_pool, qh, kh, vh, oh, lh)
+    assert torch.equal(oh, g.out.cpu())
+    assert torch.equal(lh, g.lse.cpu())
+
+
+@pytest.mark.parametrize("idx,n_random", [(4, 1024), (5, 1024)])
+def test_full_size_sampled(idx, n_random):
+    """Configurations too large for the oracle in full: gather compared in full (bit-exact V, block
+    table, exact K rows, tolerance on rotated K), attention on the first and last q tile of every
+    request plus random rows."""
+    w = wl.config(idx)
+    g = gu.run_layer(w, layer=idx)
+    assert g.status == 0
+    gu.check_placement(g)
+    gu.check_untouched(g)
+    rng = np.random.default_rng(idx)
+    reqs = range(w.batch) if idx == 4 else sorted(rng.choice(w.batch, size=8, replace=False).tolist())
+    asm, kmx, kmean = gu.check_assembled(g, requests=reqs)
+    tile_tokens = 128 // (w.shape.num_q_heads // w.shape.num_kv_heads)
+    rows = {r: gu.sample_rows(w, r, rng, n_random // len(list(reqs)), tile_tokens) for r in reqs}
+    gu.check_attention(g, asm, rows_by_request=rows)

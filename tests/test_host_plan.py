@@ -1,0 +1,108 @@
+"""CPU-only checks of the library boundary: exported symbols, host placement vs the oracle,
+and every validation error, none of which launches a kernel."""
+import copy
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import tessera_oracle as orc
+from paper_2609_32999_b200 import binding as tb
+from paper_2609_32999_b200 import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "tessera.h")).read()
+    declared = re.findall(r"TESSERA_API\s+\w+\s+(tessera_\w+)\s*\(", hdr)
+    assert len(declared) >= 11 and set(declared) == set(tb.EXPORTS)
+    lib = ctypes.CDLL(tb.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+@pytest.mark.parametrize("make", [lambda: wl.config(1), lambda: wl.config(2), lambda: wl.adversarial(),
+                                  lambda: wl.config(3), lambda: wl.config(5, requests_override=4)])
+def test_host_placement_matches_oracle(make):
+    w = make()
+    plan = tb.Plan(w, host_only=True)
+    page_off, pages, src_slot = plan.block_table()
+    st, o_off, o_pages, o_src, _ = orc.placement(w)
+    assert st == 0
+    assert np.array_equal(page_off, o_off)
+    assert np.array_equal(pages, o_pages)
+    assert np.array_equal(src_slot, o_src)
+    assert plan.info.total_tokens == w.total_tokens and plan.info.n_q == w.n_q
+    assert plan.info.cached_tokens == w.cached_tokens and plan.info.qk_pairs == w.qk_pairs
+    assert plan.info.gather_bytes == wl.gather_bytes(w) and plan.info.attn_flops == wl.attention_flops(w)
+    plan.destroy()
+
+
+def test_host_only_plan_refuses_device_calls():
+    plan = tb.Plan(wl.config(1), host_only=True)
+    with pytest.raises(tb.TesseraError) as e:
+        plan.kv_compose(None, None, stream=0)
+    assert e.value.status == tb.INVALID_ARG and "HOST_ONLY" in str(e.value)
+
+
+def _base():
+    shape = wl.ModelShape(4, 2, 64, 16, 1e4)
+    return wl.build_workload("v", shape, [[4, wl.unit(40, "a", recompute=(0, 1)), wl.unit(20, "b"), 2],
+                                          [wl.unit(20, "b", recompute=(0,)), 3]],
+                             np.random.default_rng(0))
+
+
+def _mut(**kw):
+    w = copy.deepcopy(_base())
+    for k, v in kw.items():
+        setattr(w, k, np.asarray(v, dtype=np.int32) if not isinstance(v, (int, wl.ModelShape)) else v)
+    return w
+
+
+def test_validation_errors():
+    w = _base()
+    assert tb.plan_create_status(w) == tb.OK
+    assert orc.placement(w)[0] == 0
+    # recompute positions out of order
+    rp = w.recompute_pos.copy(); rp[0], rp[1] = rp[1], rp[0]
+    assert tb.plan_create_status(_mut(recompute_pos=rp)) == tb.UNSORTED_POSITIONS
+    # a position nobody supplies: drop the first recompute row (position 0 of request 0)
+    assert tb.plan_create_status(_mut(recompute_pos=w.recompute_pos[1:],
+                                      recompute_off=w.recompute_off - np.array([0, 1, 1]))) == tb.UNCOVERED_POSITION
+    # two units on one position
+    tp = w.unit_target_pos.copy(); tp[1] -= 5
+    assert tb.plan_create_status(_mut(unit_target_pos=tp)) == tb.UNIT_OVERLAP
+    # unit leaves the request
+    tp = w.unit_target_pos.copy(); tp[1] += 100
+    assert tb.plan_create_status(_mut(unit_target_pos=tp)) == tb.UNIT_OVERLAP
+    # page ids
+    up = w.unit_pages.copy(); up[0] = w.num_pool_pages
+    assert tb.plan_create_status(_mut(unit_pages=up)) == tb.PAGE_OUT_OF_RANGE
+    fp = w.free_pages.copy(); fp[0] = w.unit_pages[0]
+    assert tb.plan_create_status(_mut(free_pages=fp)) == tb.PAGE_OUT_OF_RANGE
+    fp = w.free_pages.copy(); fp[1] = fp[0]
+    assert tb.plan_create_status(_mut(free_pages=fp)) == tb.PAGE_OUT_OF_RANGE
+    assert tb.plan_create_status(_mut(free_pages=w.free_pages[:2])) == tb.OUT_OF_PAGES
+    # malformed descriptor
+    assert tb.plan_create_status(_mut(unit_page_off=w.unit_page_off[::-1].copy())) == tb.INVALID_ARG
+    st = w.unit_cached_stride.copy(); st[0] = 2
+    assert tb.plan_create_status(_mut(unit_cached_stride=st)) == tb.INVALID_ARG
+    # shapes
+    for bad in (wl.ModelShape(4, 3, 64, 16, 1e4), wl.ModelShape(4, 2, 96, 16, 1e4), wl.ModelShape(4, 2, 64, 12, 1e4),
+                wl.ModelShape(4, 2, 64, 16, 1e4, rope_pairing=1), wl.ModelShape(64, 2, 64, 16, 1e4)):
+        assert tb.plan_create_status(_mut(shape=bad)) == tb.UNSUPPORTED_SHAPE
+    assert "page" in tb.last_error() or "head" in tb.last_error() or "group" in tb.last_error()
+
+
+def test_empty_batch_and_empty_request():
+    shape = wl.ModelShape(4, 2, 64, 16, 1e4)
+    w = wl.build_workload("empty", shape, [], np.random.default_rng(0))
+    plan = tb.Plan(w, host_only=True)
+    assert plan.info.total_tokens == 0 and plan.info.n_q == 0
+    w = wl.build_workload("one-empty", shape, [[], [3]], np.random.default_rng(0))
+    plan = tb.Plan(w, host_only=True)
+    page_off, pages, src = plan.block_table()
+    assert list(page_off) == [0, 0, 1] and list(src) == [-1, -1, -1]
