@@ -54,7 +54,8 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     const size_t o_poff = place<int32_t>(off, pl->page_off.size());
     const size_t o_pages = place<int32_t>(off, pl->pages.size());
     const size_t o_tiles = place<AttnTile>(off, pl->tiles.size());
-    const size_t o_order = place<int32_t>(off, pl->tile_order.size());
+    const size_t o_work = place<AttnWork>(off, pl->work.size());
+    const size_t o_seq = place<int32_t>(off, pl->seq_len.size());
     const size_t o_status = place<int32_t>(off, 4);
     pl->host_blob.assign(off, 0);
     char *hb = pl->host_blob.data();
@@ -69,7 +70,8 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     put(o_poff, pl->page_off.data(), pl->page_off.size() * 4);
     put(o_pages, pl->pages.data(), pl->pages.size() * 4);
     put(o_tiles, pl->tiles.data(), pl->tiles.size() * sizeof(AttnTile));
-    put(o_order, pl->tile_order.data(), pl->tile_order.size() * 4);
+    put(o_work, pl->work.data(), pl->work.size() * sizeof(AttnWork));
+    put(o_seq, pl->seq_len.data(), pl->seq_len.size() * 4);
     TS_CUDA(cudaMalloc(&d.blob, off));
     TS_CUDA(cudaMemcpyAsync(d.blob, hb, off, cudaMemcpyHostToDevice, st));
     char *db = static_cast<char *>(d.blob);
@@ -83,7 +85,8 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     d.page_off = reinterpret_cast<int32_t *>(db + o_poff);
     d.pages = reinterpret_cast<int32_t *>(db + o_pages);
     d.tiles = reinterpret_cast<AttnTile *>(db + o_tiles);
-    d.tile_order = reinterpret_cast<int32_t *>(db + o_order);
+    d.work = reinterpret_cast<AttnWork *>(db + o_work);
+    d.seq_len = reinterpret_cast<int32_t *>(db + o_seq);
     d.status = reinterpret_cast<int32_t *>(db + o_status);
     return TESSERA_OK;
 }
@@ -184,7 +187,7 @@ int32_t tessera_plan_get_info(const tessera_plan *pl, tessera_plan_info *info) {
     info->attn_flops = 4LL * pl->cfg.head_dim * pl->cfg.num_q_heads * pl->qk_pairs;
     info->n_rope_rows = (int32_t)pl->rope_delta.size();
     info->n_gather_items = (int32_t)pl->items.size();
-    info->n_attn_items = (int32_t)pl->tile_order.size();
+    info->n_attn_items = pl->attn_kernel == 1 ? (int32_t)pl->work.size() : (int32_t)(pl->n_q * pl->cfg.num_kv_heads);
     info->attn_kernel = pl->attn_kernel;
     return TESSERA_OK;
 }

@@ -218,11 +218,29 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
             t.kv_full = d->recompute_pos[j0] + 1;
             pl->tiles.push_back(t);
         }
-    pl->tile_order.resize(pl->tiles.size() * (size_t)Hkv);
-    std::iota(pl->tile_order.begin(), pl->tile_order.end(), 0);
-    std::stable_sort(pl->tile_order.begin(), pl->tile_order.end(), [&](int32_t a, int32_t b) {
-        return pl->tiles[a / Hkv].kv_len > pl->tiles[b / Hkv].kv_len;
-    });
+    // tcgen05 work items: consecutive tiles of a request share one thread block (and every K/V page
+    // they read); longest first, so that the tail of the grid is made of short items.
+    pl->work.clear();
+    {
+        const int page = B;
+        size_t first = 0;
+        while (first < pl->tiles.size()) {
+            size_t last = first;
+            while (last < pl->tiles.size() && pl->tiles[last].req == pl->tiles[first].req) ++last;
+            for (size_t k = first; k < last; k += 2) {
+                const int32_t a = (int32_t)k, b2 = (k + 1 < last) ? (int32_t)(k + 1) : -1;
+                const int steps = (pl->tiles[b2 >= 0 ? b2 : a].kv_len + page - 1) / page;
+                for (int h = 0; h < Hkv; ++h) pl->work.push_back({a, b2, h, steps});
+            }
+            first = last;
+        }
+        auto cost = [&](const AttnWork &w) {
+            int c = (pl->tiles[w.tile_a].kv_len + page - 1) / page;
+            if (w.tile_b >= 0) c += (pl->tiles[w.tile_b].kv_len + page - 1) / page;
+            return c;
+        };
+        std::stable_sort(pl->work.begin(), pl->work.end(), [&](const AttnWork &x, const AttnWork &y) { return cost(x) > cost(y); });
+    }
 
     pl->total_tokens = total;
     pl->n_q = n_q;

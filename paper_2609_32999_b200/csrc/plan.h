@@ -12,7 +12,7 @@ namespace tessera {
 
 constexpr int kGatherItemTokens = 32;   // token rows per thread block of the gather kernel
 constexpr int kAttnTileRows = 128;      // query rows (tokens x grouped heads) per tcgen05 tile
-constexpr bool kHaveTensorCoreKernel = false;
+constexpr bool kHaveTensorCoreKernel = true;
 
 // One thread block of the gather / shift kernel: `count` consecutive entries of the copy list that
 // belong to one cached unit.  Entry i uses row (row0 + i * row_step) of the cos/sin table.
@@ -26,6 +26,12 @@ struct AttnTile {
     int32_t req, q_begin, n_tok, kv_len, kv_full, pad0, pad1, pad2;
 };
 
+// One thread block of the tcgen05 attention kernel: KV head `kvh` of query tiles tile_a and tile_b
+// (consecutive tiles of one request; tile_b = -1 when the request has an odd tile left over).
+struct AttnWork {
+    int32_t tile_a, tile_b, kvh, n_steps;
+};
+
 struct DeviceTables {
     void *blob = nullptr;          // one allocation holding everything below
     int32_t *g_src = nullptr, *g_dst = nullptr;
@@ -37,7 +43,8 @@ struct DeviceTables {
     int32_t *page_off = nullptr;   // [batch+1]
     int32_t *pages = nullptr;      // block tables
     AttnTile *tiles = nullptr;
-    int32_t *tile_order = nullptr; // work items (tile * H_kv + kv head), longest first
+    AttnWork *work = nullptr;      // tcgen05 work items, longest first
+    int32_t *seq_len = nullptr;    // [batch]
     int32_t *status = nullptr;     // device status word(s)
     // staging for the host-buffer entry point (allocated on first use)
     void *st_q = nullptr, *st_k = nullptr, *st_v = nullptr, *st_o = nullptr;
@@ -62,7 +69,7 @@ struct tessera_plan {
     std::vector<int32_t> rope_delta;       // sorted distinct shift amounts
     std::vector<float> rope_table;         // [rows][D/2][2]
     std::vector<tessera::AttnTile> tiles;
-    std::vector<int32_t> tile_order;
+    std::vector<tessera::AttnWork> work;
     int32_t attn_kernel = 0;
     int32_t tile_tokens = 0;
 
