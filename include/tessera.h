@@ -182,6 +182,34 @@ TESSERA_API int32_t tessera_composed_prefill_host(tessera_plan *plan, void *k_po
                                       const void *q_host, const void *k_new_host, const void *v_new_host,
                                       void *out_host, float *lse_host, void *stream);
 
+/*
+ * In-place RoPE shift for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this is a service entry of this library.)  Some callers run where cudaMalloc is off
+ * limits: inside a serving engine that owns the whole device through its own memory pool, in a
+ * phase where the allocator must stay untouched, or under a no-allocation-after-start-up rule.
+ * tessera_plan_create allocates its tables, so such callers cannot use the plan-based shift.  This
+ * call needs no plan and allocates nothing: its cos/sin table sits in a fixed 256 KB array inside
+ * the library image, which every device that loads the library holds until the process exits.
+ *
+ * Rotates, in place, row slots[i] of k_pool (device, pool layout above) by shifts[slot_shift[i]]
+ * positions, with the arithmetic of tessera_rope_shift (cos/sin in fp64 stored as fp32, fp32 math,
+ * one round-to-nearest-even to bf16; a shift of 0 leaves the bits unchanged).
+ *   cfg        host: head_dim, num_kv_heads, rope_theta / inv_freq, rope_pairing are read
+ *   slots      device [n_slots] pool slot ids (page * page_size + offset); each listed once
+ *   slot_shift device [n_slots] index into shifts; entries outside [0, n_shifts) are skipped
+ *   shifts     host   [n_shifts] shift amounts; n_shifts <= TESSERA_STATIC_MAX_SHIFTS, otherwise
+ *              TESSERA_UNSUPPORTED_SHAPE and nothing is launched
+ * The first call on a device looks up the array's device address (once per device, with that device
+ * current); make that first call before any stream capture begins.  All calls on a device share
+ * the array and each call overwrites the rows it uses (nothing in it has to start at zero), so two
+ * calls whose GPU work can overlap - different streams without ordering - race on it; calls on one
+ * stream are safe.  Work is enqueued on `stream`; the call does not wait for it.
+ */
+#define TESSERA_STATIC_MAX_SHIFTS 512
+TESSERA_API int32_t tessera_rope_shift_static(const tessera_model_cfg *cfg, void *k_pool, const int32_t *slots,
+                                              const int32_t *slot_shift, int32_t n_slots, const int32_t *shifts,
+                                              int32_t n_shifts, void *stream);
+
 /* Copies the calling thread's last error text into buf (host); returns its length. */
 TESSERA_API int32_t tessera_last_error(char *buf, int32_t len);
 

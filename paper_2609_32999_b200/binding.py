@@ -53,7 +53,8 @@ class PlanInfo(ctypes.Structure):
 
 EXPORTS = ["tessera_plan_create", "tessera_plan_destroy", "tessera_plan_block_table", "tessera_plan_get_info",
            "tessera_plan_status", "tessera_kv_compose", "tessera_rope_shift", "tessera_partial_prefill_attn",
-           "tessera_composed_prefill_host", "tessera_last_error", "tessera_launch_count"]
+           "tessera_composed_prefill_host", "tessera_rope_shift_static", "tessera_last_error",
+           "tessera_launch_count"]
 
 _vp = ctypes.c_void_p
 _lib.tessera_plan_create.argtypes = [ctypes.POINTER(ModelCfg), ctypes.POINTER(ComposeDesc), ctypes.c_int32,
@@ -66,6 +67,8 @@ _lib.tessera_kv_compose.argtypes = [_vp, _vp, _vp, ctypes.c_uint32, _vp]
 _lib.tessera_rope_shift.argtypes = [_vp, _vp, _vp]
 _lib.tessera_partial_prefill_attn.argtypes = [_vp] * 9
 _lib.tessera_composed_prefill_host.argtypes = [_vp] * 9
+_lib.tessera_rope_shift_static.argtypes = [ctypes.POINTER(ModelCfg), _vp, _vp, _vp, ctypes.c_int32, _I32P,
+                                           ctypes.c_int32, _vp]
 _lib.tessera_last_error.argtypes = [ctypes.c_char_p, ctypes.c_int32]
 _lib.tessera_launch_count.argtypes = []
 _lib.tessera_launch_count.restype = ctypes.c_int64
@@ -185,6 +188,21 @@ class Plan:
             self.destroy()
         except Exception:
             pass
+
+
+STATIC_MAX_SHIFTS = 512
+
+
+def rope_shift_static(shape, k_pool, slots, slot_shift, shifts, stream=None, inv_freq=None) -> None:
+    """tessera_rope_shift_static: rotate the listed pool slots in place without any device
+    allocation.  `slots` / `slot_shift` are int32 device tensors, `shifts` a host int32 sequence."""
+    inv = None if inv_freq is None else np.ascontiguousarray(inv_freq, dtype=np.float64)
+    cfg = ModelCfg(shape.num_q_heads, shape.num_kv_heads, shape.head_dim, shape.page_size, float(shape.rope_theta),
+                   None if inv is None else inv.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
+                   int(shape.rope_pairing), float(shape.sm_scale))
+    sh = _arr(shifts)
+    _check(_lib.tessera_rope_shift_static(ctypes.byref(cfg), _dev(k_pool), _dev(slots), _dev(slot_shift),
+                                          int(slots.numel()), _ptr(sh), len(sh), _stream(stream)))
 
 
 def plan_create_status(w, host_only: bool = True) -> int:

@@ -9,7 +9,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtessera.so")
-SOURCES = ["api.cu", "plan.cu", "gather_rope.cu", "attn_simt.cu", "attn_tc.cu"]
+SOURCES = ["api.cu", "plan.cu", "gather_rope.cu", "attn_simt.cu", "attn_tc.cu",
+           "rope_shift_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 

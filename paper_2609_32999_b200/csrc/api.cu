@@ -116,6 +116,9 @@ int32_t attention(const tessera_plan *pl, void *k_pool, void *v_pool, const void
 
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
+// Lets entry points defined in other files record the calling thread's error text.
+int32_t api_set_error(int32_t code, const std::string &msg) { return set_error(code, msg); }
+
 }  // namespace tessera
 
 using namespace tessera;
