@@ -131,7 +131,7 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2609_32999_b200 import workloads as wl
-    w = wl.config(args.config)
+    w = wl.config(args.config, requests_override=args.requests)
     t = wl.make_tensors(w, layer=0, device="cpu")
     bits = host_bits(t)
     per_step_budget = max(2.0, min(20.0, 90.0 / max(args.steps + args.warmup, 1)))
@@ -162,6 +162,7 @@ def main():
     ap.add_argument("--steps", type=int, default=32)
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--config", type=int, default=4)
+    ap.add_argument("--requests", type=int, default=None, help="override the number of requests (profiling small cases)")
     ap.add_argument("--layers", type=int, default=4, help="distinct per-layer pools cycled through")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle attention sampling")
@@ -186,7 +187,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     # every rank owns an independent batch of the same configuration (requests do not interact)
-    w = wl.config(args.config, seed=wl.BASE_SEED + args.config + 7919 * rank)
+    w = wl.config(args.config, seed=wl.BASE_SEED + args.config + 7919 * rank, requests_override=args.requests)
     plan = tb.Plan(w)
     info = plan.info
     layers = [wl.make_tensors(w, layer=l, device=dev, seed=wl.BASE_SEED + rank) for l in range(args.layers)]

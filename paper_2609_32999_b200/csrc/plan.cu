@@ -222,7 +222,7 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
     // they read); longest first, so that the tail of the grid is made of short items.
     pl->work.clear();
     {
-        const int page = B;
+        const int page = 2 * B;      // the kernel advances two pages per step
         size_t first = 0;
         while (first < pl->tiles.size()) {
             size_t last = first;
