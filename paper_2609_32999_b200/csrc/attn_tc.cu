@@ -3,22 +3,26 @@
 //
 // One thread block works on one KV head and up to TWO query tiles of the same request (128 rows
 // each: 128/g recompute tokens x the g query heads of the group), which share every K/V page they
-// read.  A step covers 128 keys (two pages).  Warp roles:
-//   warps 0-3 / 4-7 : softmax of tile 0 / tile 1 - thread i owns accumulator row i (TMEM lane i)
-//   warp 8          : TMA producer - Q tiles once, then K and V of every step through one ring of
-//                     32 KB shared-memory slots; page ids come from the request's block table
-//   warp 9          : issues tcgen05.mma (one lane) and owns the TMEM allocation
+// read.  A step covers 128 keys (two pages).  Warp roles (384 threads):
+//   warps 0-7  : softmax.  All eight work on one tile at a time and alternate between the tiles;
+//                warps 0-3 own columns 0-63 of a row, warps 4-7 columns 64-127 (TMEM lane = row)
+//   warp 8     : TMA producer - Q tiles once, then K and V of every step through one ring of
+//                32 KB shared-memory slots; page ids come from the request's block table
+//   warp 9, 10 : issue tcgen05.mma for tile 0 / tile 1 (one lane each); warp 9 owns the TMEM allocation
+//   warp 11    : idle (completes the warp group that hands its registers to the softmax warps)
 // Per tile and step:  S = Q K^T (both operands in shared memory) -> 128 fp32 TMEM columns;
-// softmax reads S, writes P as bf16 over the first 64 of those columns; O += P V takes P straight
-// from TMEM, so probabilities never touch shared memory.  The MMA warp issues P.V of step j and
-// then S of step j+1 of the same tile; while one tile is in softmax the tensor pipe works for the
-// other.  Pages past a tile's last query position are never loaded; only steps that cross some
-// row's causal limit are masked.  The running maximum is refreshed only when it grows by more than
-// 2^8, so the accumulator in TMEM is rescaled rarely.  Every wait is bounded (ptx::mbar_wait).
+// softmax reads S and writes P as bf16 back over part of those columns; O += P V takes P straight
+// from TMEM, so probabilities never touch shared memory.  Each issuing warp sends P.V of step j and
+// then S of step j+1 of its tile; while the softmax warps are on one tile the tensor pipe works
+// for the other.  Pages past a tile's last query position are never loaded; only steps that cross
+// some row's causal limit are masked.  Probabilities are taken against a reference maximum that is
+// refreshed only when a row's partial sum would exceed 2^8, so the accumulator in TMEM is rescaled
+// rarely.  Every wait is bounded (ptx::mbar_wait).
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdio>
 
 #include "launch.h"
 #include "plan.h"
@@ -34,8 +38,12 @@ constexpr int kD = 128;            // head_dim
 constexpr int kPage = 64;          // page size
 constexpr int kStep = 128;         // keys per step (two pages)
 constexpr int kRows = 128;         // rows per query tile
+#ifdef TESSERA_ATTN_TRACE
+constexpr int kRing = 4;
+#else
 constexpr int kRing = 5;           // K/V ring slots
-constexpr int kThreads = 320;
+#endif
+constexpr int kThreads = 384;        // 8 softmax warps, producer, MMA, 2 idle warps (register donors)
 
 constexpr uint32_t kQTileBytes = kRows * kD * 2;         // 32 KB: [d half][128 rows][128 B]
 constexpr uint32_t kSlotBytes = kStep * kD * 2;          // 32 KB: [d half][128 keys][128 B]
@@ -50,7 +58,6 @@ constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemS = 0;      // S[tile] at tile * 128 (P[tile] = its first 64 columns)
 constexpr uint32_t kTmemO = 256;    // O[tile] at 256 + tile * 128
 
-constexpr float kRescaleThreshold = 8.f;   // log2 units
 
 struct Barriers {
     uint64_t q_full[2];
@@ -71,6 +78,16 @@ __device__ __forceinline__ void fma2(float &d0, float &d1, float a0, float a1, f
         " fma.rn.f32x2 rd, ra, rb, rc;\n mov.b64 {%0, %1}, rd;\n}"
         : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b), "f"(c));
 }
+template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+__device__ __forceinline__ void named_sync(int id, int count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+// (a0, a1) += (b0, b1) with one packed instruction.
+__device__ __forceinline__ void add2(float &a0, float &a1, float b0, float b1) {
+    asm("{\n .reg .b64 ra, rb;\n mov.b64 ra, {%0, %1};\n mov.b64 rb, {%2, %3};\n add.rn.f32x2 ra, ra, rb;\n mov.b64 {%0, %1}, ra;\n}"
+        : "+f"(a0), "+f"(a1) : "f"(b0), "f"(b1));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -89,6 +106,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     __shared__ __align__(8) Barriers bars;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
+    __shared__ float s_xchg[2][kRows];              // row maxima exchanged between the two column halves
+    __shared__ int s_flag[2][2][4][2];              // [step parity][tile][warp pair][half]
+#ifdef TESSERA_ATTN_TRACE
+    __shared__ unsigned s_trace[2][16][8];
+    __shared__ unsigned s_ptrace[16][4];
+#define TRACE(q, j, e) do { if ((j) >= 8 && (j) < 24) s_trace[q][(j) - 8][e] = (unsigned)clock64(); } while (0)
+#define PTRACE(j, e) do { if ((j) >= 8 && (j) < 24) s_ptrace[(j) - 8][e] = (unsigned)clock64(); } while (0)
+#else
+#define TRACE(q, j, e) do {} while (0)
+#define PTRACE(j, e) do {} while (0)
+#endif
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const AttnWork wk = work[blockIdx.x];
@@ -108,12 +136,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bars.q_full[i]), 1);
             mbar_init(smem_u32(&bars.s_full[i]), 1);
-            mbar_init(smem_u32(&bars.p_full[i]), kRows);
+            mbar_init(smem_u32(&bars.p_full[i]), 2 * kRows);
             mbar_init(smem_u32(&bars.pv_done[i]), 1);
         }
         for (int i = 0; i < kRing; ++i) {
             mbar_init(smem_u32(&bars.full[i]), 1);
-            mbar_init(smem_u32(&bars.empty[i]), 1);
+            mbar_init(smem_u32(&bars.empty[i]), n_tiles);
         }
         fence_barrier_init();
     }
@@ -132,6 +160,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const uint32_t tmem = s_tmem_base;
     volatile int *abort_flag = &s_abort;
 
+    // Registers move from the producer / MMA warp group to the softmax warps, which hold a whole
+    // 128-column row of S plus the packed probabilities.
+    if (warp >= 8) {
+    reg_dealloc<56>();
     if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -158,7 +190,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 #pragma unroll
                     for (int kv = 0; kv < 2; ++kv) {
                         const int item = 2 * j + kv, slot = item % kRing;
+                        PTRACE(j, 2 * kv);
                         mbar_wait(smem_u32(&bars.empty[slot]), ((item / kRing) & 1) ^ 1, abort_flag, status, 1 + kv);
+                        PTRACE(j, 2 * kv + 1);
                         const uint32_t fb = smem_u32(&bars.full[slot]);
                         mbar_expect_tx(fb, kSlotBytes);
                         const uint32_t dst = smem_u32(sm + kSmemRing + slot * kSlotBytes);
@@ -172,175 +206,227 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 __syncwarp();
             }
         }
-    } else if (warp == 9) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == 9 || (warp == 10 && n_tiles == 2)) {
+        // ------------------------------------------------------------------ MMA issuers: warp 9 for
+        // tile 0, warp 10 for tile 1.  Each runs its own tile's chain, so the waits of one overlap
+        // the MMAs of the other; a ring slot is free again once both have released it.
         constexpr uint32_t idesc_s = idesc_bf16(kRows, kStep, false);
         constexpr uint32_t idesc_o = idesc_bf16(kRows, kD, true);
+        const int q = warp - 9;
+        const int my_steps = q ? n_steps1 : n_steps0;
         const int tail_step = (T % kStep) ? T / kStep : -1;        // step holding slots past the sequence end
+        const uint32_t qbase = smem_u32(sm + kSmemQ + q * kQTileBytes);
+        const uint32_t tS = tmem + kTmemS + q * 128, tO = tmem + kTmemO + q * 128;
 
         auto ring_wait = [&](int item, int code) {
             mbar_wait(smem_u32(&bars.full[item % kRing]), (item / kRing) & 1, abort_flag, status, code);
             tc_fence_after();
         };
-        auto issue_s = [&](int q, int j) {                         // S[q] = Q_q K_j^T (lane 0)
+        auto issue_s = [&](int j) {                                // S[q] = Q_q K_j^T (lane 0)
             const uint32_t kbase = smem_u32(sm + kSmemRing + ((2 * j) % kRing) * kSlotBytes);
-            const uint32_t qbase = smem_u32(sm + kSmemQ + q * kQTileBytes);
-            const uint32_t d = tmem + kTmemS + q * 128;
 #pragma unroll
             for (int k = 0; k < kD / 16; ++k) {
                 const uint64_t a = smem_desc_sw128(qbase + (k / 4) * (kQTileBytes / 2) + (k % 4) * 32, 16, 1024);
                 const uint64_t b = smem_desc_sw128(kbase + (k / 4) * kHalfBytes + (k % 4) * 32, 16, 1024);
-                umma_ss(d, a, b, idesc_s, k > 0);
+                umma_ss(tS, a, b, idesc_s, k > 0);
             }
             umma_commit(smem_u32(&bars.s_full[q]));
+            umma_commit(smem_u32(&bars.empty[(2 * j) % kRing]));   // K_j no longer needed by this tile
         };
 
-        for (int q = 0; q < n_tiles; ++q) mbar_wait(smem_u32(&bars.q_full[q]), 0, abort_flag, status, 4);
+        mbar_wait(smem_u32(&bars.q_full[q]), 0, abort_flag, status, 4);
         ring_wait(0, 3);
-        if (lane == 0) {
-            for (int q = 0; q < n_tiles; ++q) issue_s(q, 0);
-            umma_commit(smem_u32(&bars.empty[0]));
-        }
+        if (lane == 0) issue_s(0);
         __syncwarp();
         for (int j = 0; j < n_steps; ++j) {
+            if (lane == 0 && q == 0) TRACE(0, j, 7);
             ring_wait(2 * j + 1, 5);                               // V_j
             const int vslot = (2 * j + 1) % kRing;
+            const bool more = j + 1 < n_steps;
+            if (j >= my_steps) {
+                // this tile is finished (tile 0 may need fewer steps): only release the slots
+                if (more) ring_wait(2 * j + 2, 3);
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&bars.empty[vslot]));
+                    if (more) mbar_arrive(smem_u32(&bars.empty[(2 * j + 2) % kRing]));
+                }
+                __syncwarp();
+                continue;
+            }
             if (j == tail_step) {
                 // V rows past the end of the sequence hold whatever the page held before; their
-                // probabilities are zero, but 0 x NaN would still poison the accumulator.
+                // probabilities are zero, but 0 x NaN would still poison the accumulator.  (Both
+                // issuing warps may write these zeros; the values agree.)
                 uint8_t *v = sm + kSmemRing + vslot * kSlotBytes;
                 for (int r = T - j * kStep; r < kStep; ++r)
                     if (lane < 16) *reinterpret_cast<uint4 *>(v + (lane >> 3) * kHalfBytes + r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
                 fence_proxy_async_smem();
                 __syncwarp();
             }
-            const bool more = j + 1 < n_steps;
+            const bool next_s = j + 1 < my_steps;
             if (more) ring_wait(2 * j + 2, 3);                     // K_{j+1}
+            if (lane == 0 && q == 0) TRACE(1, j, 7);
             const uint32_t vbase = smem_u32(sm + kSmemRing + vslot * kSlotBytes);
-            for (int q = 0; q < n_tiles; ++q) {
-                const int my_steps = q ? n_steps1 : n_steps0;
-                if (j >= my_steps) continue;
-                mbar_wait(smem_u32(&bars.p_full[q]), j & 1, abort_flag, status, 6);
-                tc_fence_after();
-                if (lane == 0) {
-                    const uint32_t d = tmem + kTmemO + q * 128;
-                    const uint32_t p = tmem + kTmemS + q * 128;
-#pragma unroll
-                    for (int k = 0; k < kStep / 16; ++k) {
-                        const uint64_t b = smem_desc_sw128(vbase + k * 2048, kHalfBytes, 1024);
-                        umma_ts(d, p + k * 8, b, idesc_o, (j > 0) || (k > 0));
-                    }
-                    umma_commit(smem_u32(&bars.pv_done[q]));
-                    if (j + 1 < my_steps) issue_s(q, j + 1);
-                }
-                __syncwarp();
-            }
+            if (lane == 0) TRACE(q, j, 4);
+            mbar_wait(smem_u32(&bars.p_full[q]), j & 1, abort_flag, status, 6);
+            tc_fence_after();
             if (lane == 0) {
+                TRACE(q, j, 5);
+#pragma unroll
+                for (int k = 0; k < kStep / 16; ++k) {
+                    const uint64_t b = smem_desc_sw128(vbase + k * 2048, kHalfBytes, 1024);
+                    umma_ts(tO, tS + (k >> 2) * 64 + (k & 3) * 8, b, idesc_o, (j > 0) || (k > 0));
+                }
+                umma_commit(smem_u32(&bars.pv_done[q]));
                 umma_commit(smem_u32(&bars.empty[vslot]));
-                if (more) umma_commit(smem_u32(&bars.empty[(2 * j + 2) % kRing]));
+                if (next_s) issue_s(j + 1);
+                else if (more) mbar_arrive(smem_u32(&bars.empty[(2 * j + 2) % kRing]));
+                TRACE(q, j, 6);
             }
             __syncwarp();
         }
+    }
     } else {
+        reg_alloc<224>();
         // ------------------------------------------------------------------ softmax + epilogue
-        const int q = warp >> 2;                       // tile handled by this warp group
-        if (q < n_tiles) {
+        // All eight warps work on ONE tile at a time and alternate between the tiles: warps 0-3 take
+        // columns 0-63 of a row, warps 4-7 columns 64-127 (warp w and w + 4 share TMEM lanes).  The
+        // two threads of a row keep identical reference maxima and separate partial sums.
+        const int h = warp >> 2;                       // column half
+        const int pair = warp & 3;                     // named barrier 1 + pair joins warps w and w + 4
+        const int row = tid & 127;
+        const uint32_t lane_base = (uint32_t)(pair * 32) << 16;
+        int tok[2], p_row[2];
+        bool row_valid[2];
+        float m_row[2] = {-INFINITY, -INFINITY}, l_row[2] = {0.f, 0.f};
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
             const AttnTile &t = q ? t1 : t0;
-            const int my_steps = q ? n_steps1 : n_steps0;
-            const int row = tid & 127;
-            const int tok = min(row / g, t.n_tok - 1);
-            const bool row_valid = row / g < t.n_tok;
-            const int p_row = q_pos[t.q_begin + tok];
-            const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-            const uint32_t tS = tmem + kTmemS + q * 128 + lane_base;
-            const uint32_t tO = tmem + kTmemO + q * 128 + lane_base;
-            float m_row = -INFINITY, l_row = 0.f;
+            tok[q] = min(row / g, t.n_tok - 1);
+            row_valid[q] = row / g < t.n_tok;
+            p_row[q] = q_pos[t.q_begin + tok[q]];
+        }
 
-            for (int j = 0; j < my_steps; ++j) {
+        for (int j = 0; j < n_steps; ++j) {
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                if (q >= n_tiles || j >= (q ? n_steps1 : n_steps0)) continue;
+                const uint32_t tS = tmem + kTmemS + q * 128 + h * 64 + lane_base;
                 // S_j complete; this also means P.V of step j-1 has completed (it was issued earlier)
+                if (tid == 0) TRACE(q, j, 0);
                 mbar_wait(smem_u32(&bars.s_full[q]), j & 1, abort_flag, status, 7);
                 tc_fence_after();
-                const int key0 = j * kStep;
-                const bool masked = key0 + kStep > t.kv_full;   // some row's causal limit falls in this step
+                if (tid == 0) TRACE(q, j, 1);
+                const int key0 = j * kStep + h * 64;
+                const bool masked = j * kStep + kStep > (q ? t1.kv_full : t0.kv_full);   // a causal limit falls in this step
+                const int pr = p_row[q];
 
-                // pass 1: row maximum
-                float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t s[32];
-                    tmem_ld32(tS + c * 32, s);
+                uint32_t pk[32];
+                float sum = 0.f, mx = -INFINITY;
+                // One pass over this thread's 64 columns: the maximum (with_max) and / or the
+                // probabilities against the current reference maximum (with_exp).
+                auto pass = [&](bool with_max, bool with_exp) {
+                    uint32_t s[64];
+                    tmem_ld32(tS, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+                    tmem_ld32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
                     tmem_wait_ld();
                     if (masked) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (key0 + c * 32 + i > p_row) s[i] = 0xff800000u;   // -inf
+                        for (int i = 0; i < 64; ++i)
+                            if (key0 + i > pr) s[i] = 0xff800000u;   // -inf
                     }
+                    if (with_max) {
+                        float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mxa[i & 3] = fmaxf(mxa[i & 3], __uint_as_float(s[i]));
+                        for (int i = 0; i < 32; ++i)
+                            mxa[i & 3] = fmaxf(mxa[i & 3], fmaxf(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])));
+                        mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
+                    }
+                    if (with_exp) {
+                        float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+                        const float neg_m = -m_row[q];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            float x0, x1;
+                            fma2(x0, x1, __uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]), scale_log2, neg_m);
+                            const float e0 = ex2(x0), e1 = ex2(x1);
+                            add2(sa[i & 3], sb[i & 3], e0, e1);
+                            pk[i] = pack_bf16(e0, e1);
+                        }
+                        sum = ((sa[0] + sb[0]) + (sa[1] + sb[1])) + ((sa[2] + sb[2]) + (sa[3] + sb[3]));
+                    }
+                };
+
+                // Fast path: probabilities against the current reference maximum.  While a thread's
+                // sum stays below 2^8 every probability does too and the reference is good enough;
+                // otherwise (and on the first step) the row takes the step's true maximum and redoes P.
+                bool stale = true;
+                if (j > 0) {
+                    pass(false, true);
+                    stale = !(sum <= 256.f);
                 }
-                const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
-                const float mc = fmaxf(m_row, mx * scale_log2);
+                // both halves of a row must take the same decision
+                const int par = j & 1;
+                const bool warp_stale = __any_sync(0xffffffffu, stale);
+                if (lane == 0) s_flag[par][q][pair][h] = warp_stale ? 1 : 0;
+                named_sync(1 + pair, 64);
+                const bool redo = (s_flag[par][q][pair][0] | s_flag[par][q][pair][1]) != 0;
                 float factor = 1.f;
-                bool rescale = false;
-                if (mc > m_row + kRescaleThreshold) {  // also true on the first step (m_row = -inf)
-                    factor = ex2(m_row - mc);          // 0 on the first step
-                    m_row = mc;
-                    rescale = j > 0;
-                }
-                if (__any_sync(0xffffffffu, rescale)) {
+                if (redo) {
+                    pass(true, false);
+                    s_xchg[h][row] = mx;
+                    named_sync(1 + pair, 64);
+                    const float mc = fmaxf(m_row[q], fmaxf(mx, s_xchg[h ^ 1][row]) * scale_log2);
+                    factor = ex2(m_row[q] - mc);       // 0 on the first step (m_row = -inf)
+                    m_row[q] = mc;
+                    named_sync(1 + pair, 64);          // s_xchg may be rewritten after this point
+                    if (j > 0) {
+                        const uint32_t tO = tmem + kTmemO + q * 128 + h * 64 + lane_base;
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t o[32];
-                        tmem_ld32(tO + c * 32, o);
-                        tmem_wait_ld();
+                        for (int c = 0; c < 2; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c * 32, o);
+                            tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-                        tmem_st32(tO + c * 32, o);
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+                            tmem_st32(tO + c * 32, o);
+                        }
                     }
+                    pass(false, true);
                 }
-
-                // pass 2: probabilities, written as bf16 over the first 64 columns of S
-                float suma[4] = {0.f, 0.f, 0.f, 0.f};
-                const float neg_m = -m_row;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t s[32];
-                    tmem_ld32(tS + c * 32, s);
-                    tmem_wait_ld();
-                    if (masked) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (key0 + c * 32 + i > p_row) s[i] = 0xff800000u;
-                    }
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        float x0, x1;
-                        fma2(x0, x1, __uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]), scale_log2, neg_m);
-                        const float a = ex2(x0), b = ex2(x1);
-                        suma[i & 3] += a + b;
-                        pk[i] = pack_bf16(a, b);
-                    }
-                    tmem_st16(tS + c * 16, pk);
-                }
-                l_row = l_row * factor + ((suma[0] + suma[1]) + (suma[2] + suma[3]));
+                if (tid == 0) TRACE(q, j, 2);
+                l_row[q] = l_row[q] * factor + sum;
+                // P as bf16 over the first 32 of this thread's 64 S columns
+                tmem_st16(tS, &pk[0]);
+                tmem_st16(tS + 16, &pk[16]);
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars.p_full[q]));
+                if (tid == 0) TRACE(q, j, 3);
             }
+        }
 
-            // epilogue: O / l -> bf16, LSE
-            mbar_wait(smem_u32(&bars.pv_done[q]), (my_steps - 1) & 1, abort_flag, status, 9);
-            tc_fence_after();
-            const float inv = 1.f / l_row;
+        // epilogue: O / l -> bf16, LSE.  Both tiles' last MMAs are complete before the shared-memory
+        // ring (idle by then) is reused to add up the two partial sums of every row.
+        for (int q = 0; q < n_tiles; ++q)
+            mbar_wait(smem_u32(&bars.pv_done[q]), ((q ? n_steps1 : n_steps0) - 1) & 1, abort_flag, status, 9);
+        tc_fence_after();
+        float *l_xchg = reinterpret_cast<float *>(sm + kSmemRing);           // [tile][half][row]
+        for (int q = 0; q < n_tiles; ++q) l_xchg[(q * 2 + h) * 128 + row] = l_row[q];
+        named_sync(1 + pair, 64);
+        for (int q = 0; q < n_tiles; ++q) {
+            const AttnTile &t = q ? t1 : t0;
+            const float l_tot = l_row[q] + l_xchg[(q * 2 + (h ^ 1)) * 128 + row];
+            const float inv = 1.f / l_tot;
             const int head = kvh * g + row % g;
-            __nv_bfloat16 *orow = out + ((size_t)(t.q_begin + tok) * H_q + head) * kD;
+            __nv_bfloat16 *orow = out + ((size_t)(t.q_begin + tok[q]) * H_q + head) * kD + h * 64;
+            const uint32_t tO = tmem + kTmemO + q * 128 + h * 64 + lane_base;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t o[32];
                 tmem_ld32(tO + c * 32, o);
                 tmem_wait_ld();
-                if (row_valid) {
+                if (row_valid[q]) {
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
                         uint32_t w[4];
@@ -351,8 +437,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     }
                 }
             }
-            if (lse && row_valid)
-                lse[(size_t)(t.q_begin + tok) * H_q + head] = (m_row + log2f(l_row)) * 0.6931471805599453f;
+            if (lse && row_valid[q] && h == 0)
+                lse[(size_t)(t.q_begin + tok[q]) * H_q + head] = (m_row[q] + log2f(l_tot)) * 0.6931471805599453f;
         }
     }
 
@@ -362,6 +448,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
+#ifdef TESSERA_ATTN_TRACE
+    if (blockIdx.x == 0 && tid == 0) {
+        const unsigned t0 = s_trace[0][0][0];
+        for (int j = 0; j < 16; ++j) {
+            for (int qq = 0; qq < 2; ++qq)
+                printf("j %d q %d | sm: wait %u got %u exp %u arr %u | mma: wait %u got %u issued %u\n", j + 8, qq,
+                       s_trace[qq][j][0] - t0, s_trace[qq][j][1] - t0, s_trace[qq][j][2] - t0, s_trace[qq][j][3] - t0,
+                       s_trace[qq][j][4] - t0, s_trace[qq][j][5] - t0, s_trace[qq][j][6] - t0);
+            printf("   mma ring: begin %u done %u | producer K: wait %u issue %u  V: wait %u issue %u\n", s_trace[0][j][7] - t0,
+                   s_trace[1][j][7] - t0, s_ptrace[j][0] - t0, s_ptrace[j][1] - t0, s_ptrace[j][2] - t0, s_ptrace[j][3] - t0);
+        }
+    }
+#endif
     if (warp == 9) tmem_dealloc(tmem, kTmemCols);
 }
 
