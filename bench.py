@@ -124,6 +124,25 @@ def host_bits(t):
     return tuple(orc.bits(x) for x in (t.k_pool, t.v_pool, t.q, t.k_new, t.v_new))
 
 
+def rank_workload(config: int, rank: int, requests=None):
+    """Every rank owns an independent batch of the same configuration: requests never interact
+    (no cross-request attention), so the path shards by request with no data-path collective."""
+    from paper_2609_32999_b200 import workloads as wl
+    return wl.config(config, seed=wl.BASE_SEED + config + 7919 * rank, requests_override=requests)
+
+
+def aggregate(times_ms, tokens, world: int, device: str):
+    """Max over ranks of every timing and sum over ranks of the tokens processed."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    n = torch.tensor([float(tokens)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return t.tolist(), n.item()
+
+
 def run_reference(args):
     """The reference arm: the oracle on the host cores, on the same workload and metric.  Each step is
     a bounded sample (a fixed share of one layer), extrapolated to a whole layer."""
@@ -186,8 +205,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    # every rank owns an independent batch of the same configuration (requests do not interact)
-    w = wl.config(args.config, seed=wl.BASE_SEED + args.config + 7919 * rank, requests_override=args.requests)
+    w = rank_workload(args.config, rank, args.requests)
     plan = tb.Plan(w)
     info = plan.info
     layers = [wl.make_tensors(w, layer=l, device=dev, seed=wl.BASE_SEED + rank) for l in range(args.layers)]
@@ -253,13 +271,7 @@ def main():
     barrier()
     e2e_ms = ea.elapsed_time(eb) / e2e_steps
 
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    toks = torch.tensor([float(w.total_tokens)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-        dist.all_reduce(toks, op=dist.ReduceOp.SUM)
-    total_ms_max, e2e_ms_max = times.tolist()
-    all_tokens = toks.item()
+    (total_ms_max, e2e_ms_max), all_tokens = aggregate([total_ms, e2e_ms], w.total_tokens, world, dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
