@@ -25,6 +25,11 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM traffic per launch of the two main kernels on config 4, from the ncu capture summarised under
+# profiles/ (one request captured; a full launch is `requests` times that, traffic grows with the
+# number of requests because requests share nothing).  Bytes per request per launch.
+NCU_TRAFFIC_PER_REQUEST_C4 = {"attn": 266.8e6 + 13.4e6, "gather": 134.5e6 + 78.3e6}
+
 METRIC = "composed_prefill_tokens_per_s_per_layer"
 UNIT = "tokens/s"
 
@@ -50,7 +55,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -305,11 +310,14 @@ def main():
                      "achieved": attn_tflops, "peak": tensor_peak, "unit": "TFLOP/s",
                      "frac": attn_tflops / tensor_peak, "peak_source": peaks["source"] + " sustained bf16 GEMM",
                      "frac_of_burst": attn_tflops / peaks["bf16_tflops"], "frac_of_nominal_2250": attn_tflops / 2250.0,
-                     "ms_per_launch": attn_ms, "flops_per_launch": int(info.attn_flops), "traffic": None},
+                     "ms_per_launch": attn_ms, "flops_per_launch": int(info.attn_flops),
+                     "traffic": NCU_TRAFFIC_PER_REQUEST_C4["attn"] * w.batch if args.config == 4 else None,
+                     "traffic_note": "DRAM bytes per launch: ncu capture of one request x requests (profiles/)"},
         "roofline_gather": {"kernel": "kv_compose (gather + RoPE shift)", "bound": "hbm", "achieved": gather_gbs,
                             "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gather_gbs / peaks["hbm_gbs"],
                             "peak_source": peaks["source"] + " copy", "frac_of_nominal_8000": gather_gbs / 8000.0,
-                            "ms_per_launch": gather_ms, "bytes_per_launch": int(info.gather_bytes), "traffic": None},
+                            "ms_per_launch": gather_ms, "bytes_per_launch": int(info.gather_bytes),
+                            "traffic": NCU_TRAFFIC_PER_REQUEST_C4["gather"] * w.batch if args.config == 4 else None},
         "recompute_tokens_per_s": w.n_q * world / (ms_per_step / 1e3),
     }
     if not args.no_cpu_baseline:
