@@ -111,11 +111,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 #ifdef TESSERA_ATTN_TRACE
     __shared__ unsigned s_trace[2][16][8];
     __shared__ unsigned s_ptrace[16][4];
+    __shared__ unsigned s_strace[2][16][4];
+#define STRACE(q, j, e) do { if ((j) >= 8 && (j) < 24) s_strace[q][(j) - 8][e] = (unsigned)clock64(); } while (0)
 #define TRACE(q, j, e) do { if ((j) >= 8 && (j) < 24) s_trace[q][(j) - 8][e] = (unsigned)clock64(); } while (0)
 #define PTRACE(j, e) do { if ((j) >= 8 && (j) < 24) s_ptrace[(j) - 8][e] = (unsigned)clock64(); } while (0)
 #else
 #define TRACE(q, j, e) do {} while (0)
 #define PTRACE(j, e) do {} while (0)
+#define STRACE(q, j, e) do {} while (0)
 #endif
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -330,6 +333,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     tmem_ld32(tS, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
                     tmem_ld32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
                     tmem_wait_ld();
+                    if (tid == 0) STRACE(q, j, 0);
                     if (masked) {
 #pragma unroll
                         for (int i = 0; i < 64; ++i)
@@ -365,12 +369,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     pass(false, true);
                     stale = !(sum <= 256.f);
                 }
+                if (tid == 0) STRACE(q, j, 1);
                 // both halves of a row must take the same decision
                 const int par = j & 1;
                 const bool warp_stale = __any_sync(0xffffffffu, stale);
                 if (lane == 0) s_flag[par][q][pair][h] = warp_stale ? 1 : 0;
                 named_sync(1 + pair, 64);
                 const bool redo = (s_flag[par][q][pair][0] | s_flag[par][q][pair][1]) != 0;
+                if (tid == 0) STRACE(q, j, 2);
                 float factor = 1.f;
                 if (redo) {
                     pass(true, false);
@@ -456,6 +462,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 printf("j %d q %d | sm: wait %u got %u exp %u arr %u | mma: wait %u got %u issued %u\n", j + 8, qq,
                        s_trace[qq][j][0] - t0, s_trace[qq][j][1] - t0, s_trace[qq][j][2] - t0, s_trace[qq][j][3] - t0,
                        s_trace[qq][j][4] - t0, s_trace[qq][j][5] - t0, s_trace[qq][j][6] - t0);
+            for (int qq = 0; qq < 2; ++qq) printf("   sm q%d: ld done %u compute done %u exchanged %u\n", qq, s_strace[qq][j][0] - t0, s_strace[qq][j][1] - t0, s_strace[qq][j][2] - t0);
             printf("   mma ring: begin %u done %u | producer K: wait %u issue %u  V: wait %u issue %u\n", s_trace[0][j][7] - t0,
                    s_trace[1][j][7] - t0, s_ptrace[j][0] - t0, s_ptrace[j][1] - t0, s_ptrace[j][2] - t0, s_ptrace[j][3] - t0);
         }
