@@ -5,6 +5,7 @@
 #include <cmath>
 #include <cstdio>
 #include <numeric>
+#include <tuple>
 
 #include <vector_types.h>
 
@@ -239,7 +240,16 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
             if (w.tile_b >= 0) c += (pl->tiles[w.tile_b].kv_len + page - 1) / page;
             return c;
         };
-        std::stable_sort(pl->work.begin(), pl->work.end(), [&](const AttnWork &x, const AttnWork &y) { return cost(x) > cost(y); });
+        // Longest first in coarse cost bands; inside a band, items of one (request, KV head) stay
+        // together, so thread blocks that run at the same time stream the same K/V pages and find
+        // them in L2.
+        int max_cost = 1;
+        for (const AttnWork &w : pl->work) max_cost = std::max(max_cost, cost(w));
+        const int band = std::max(1, max_cost / kAttnCostBands);
+        auto key = [&](const AttnWork &w) {
+            return std::make_tuple(-(cost(w) / band), pl->tiles[w.tile_a].req, w.kvh, -cost(w));
+        };
+        std::stable_sort(pl->work.begin(), pl->work.end(), [&](const AttnWork &x, const AttnWork &y) { return key(x) < key(y); });
     }
 
     pl->total_tokens = total;

@@ -13,6 +13,7 @@ namespace tessera {
 constexpr int kGatherItemTokens = 32;   // token rows per thread block of the gather kernel
 constexpr int kAttnTileRows = 128;      // query rows (tokens x grouped heads) per tcgen05 tile
 constexpr bool kHaveTensorCoreKernel = true;
+constexpr int kAttnCostBands = 16;      // cost bands of the attention work list (longest band first)
 
 // One thread block of the gather / shift kernel: `count` consecutive entries of the copy list that
 // belong to one cached unit.  Entry i uses row (row0 + i * row_step) of the cos/sin table.
