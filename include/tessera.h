@@ -86,6 +86,15 @@ typedef struct tessera_compose_desc {
     const int32_t *recompute_pos;       /* query rows: positions, strictly ascending per request      */
     const int32_t *free_pages;          /* destination page ids, consumed in order, request by request */
     int32_t n_free;
+    /* Optional (NULL = default), used to RETAIN freshly computed units in reusable form (Sec. 5.3: the
+       miss prefill keeps an unrotated copy for the cache; Sec. 6.1: pre-RoPE keys are captured): */
+    const int32_t *unit_src_offset;     /* [n_units] offset (0 .. page_size-1) of the unit's token 0 inside
+                                           its first source page; default 0.  Lets a unit be read out of the
+                                           middle of another request's pages; it then spans
+                                           ceil((offset + len) / page_size) source pages                 */
+    const int32_t *unit_target_stride;  /* [n_units] 1 (default): token i is rotated for position
+                                           target_pos + i; 0: every token is rotated for position
+                                           target_pos (with target_pos = 0: written without rotation)     */
 } tessera_compose_desc;
 
 typedef struct tessera_plan tessera_plan;
@@ -147,6 +156,8 @@ TESSERA_API int32_t tessera_plan_status(tessera_plan *plan, int32_t *detail, voi
  * their cached position to their new position on the way (fp32 math, one round-to-nearest-even to
  * bf16; a shift of 0 is a bit copy); without it K rows are bit copies and tessera_rope_shift must
  * follow.  k_pool, v_pool: device, layout above; source and destination pages live in the same pool.
+ * The same call retains units: a plan whose "requests" are cache entries, whose sources are the pages
+ * of a finished request (unit_src_offset) and whose unit_target_stride is 0 writes the un-rotated form.
  */
 TESSERA_API int32_t tessera_kv_compose(const tessera_plan *plan, void *k_pool, void *v_pool, uint32_t flags, void *stream);
 

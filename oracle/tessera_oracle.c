@@ -53,6 +53,7 @@ int oracle_placement(int batch, const int32_t *seq_len, const int32_t *unit_off,
                      const int32_t *unit_page_off, const int32_t *unit_pages,
                      const int32_t *recompute_off, const int32_t *recompute_pos,
                      const int32_t *free_pages, int n_free, int page_size,
+                     const int32_t *unit_src_offset /* nullable: 0 */,
                      int32_t *page_off, int32_t *pages, int32_t *src_slot, int32_t *fresh_idx)
 {
     int next_free = 0;
@@ -73,7 +74,8 @@ int oracle_placement(int batch, const int32_t *seq_len, const int32_t *unit_off,
                 if (p < 0 || p >= T) return -2;
                 if (!cached) continue;
                 if (src_slot[tok_base + p] != -1) return -3;            /* two units on one position */
-                src_slot[tok_base + p] = unit_pages[unit_page_off[u] + i / page_size] * page_size + i % page_size;
+                int si = i + (unit_src_offset ? unit_src_offset[u] : 0);   /* token index inside the source pages */
+                src_slot[tok_base + p] = unit_pages[unit_page_off[u] + si / page_size] * page_size + si % page_size;
             }
         }
         for (int j = recompute_off[r]; j < recompute_off[r + 1]; ++j) {
@@ -117,7 +119,10 @@ void oracle_rope_rotate(const double *x, double *out, int D, double delta, doubl
  *   recomputed position j  -> K = k_new[j], V = v_new[j] (bit copies);
  *   otherwise, cached unit u at offset i = p - target_pos(u):
  *        V = pool row (bit copy: values carry no rotation),
- *        K = pool row rotated by delta = p - (cached_pos(u) + stride(u) * i).
+ *        K = pool row rotated by delta = (target_pos(u) + tstride(u) * i) - (cached_pos(u) + stride(u) * i),
+ *            tstride = 1 unless given (0 = every token rotated for position target_pos(u): the form in
+ *            which a freshly computed unit is retained when target_pos = 0, Sec. 5.3 / 6.1);
+ *        the unit's token i sits at source slot (src_offset(u) + i) of its pages (src_offset 0 unless given).
  * k_asm is fp64 and left unrounded.  k_bits / k_exact: rows whose result is a bit
  * copy (recomputed rows and delta == 0) are given as bf16 bits with k_exact = 1.
  * ------------------------------------------------------------------------- */
@@ -129,6 +134,7 @@ int oracle_assemble(int r, const int32_t *seq_len, const int32_t *unit_off,
                     int page_size, int H_kv, int D, double theta, const double *inv_freq, int pairing,
                     const uint16_t *k_pool, const uint16_t *v_pool,
                     const uint16_t *k_new, const uint16_t *v_new,
+                    const int32_t *unit_src_offset /* nullable */, const int32_t *unit_target_stride /* nullable */,
                     double *k_asm, uint16_t *v_asm, uint16_t *k_bits, uint8_t *k_exact, int32_t *delta_out)
 {
     int T = seq_len[r];
@@ -140,8 +146,10 @@ int oracle_assemble(int r, const int32_t *seq_len, const int32_t *unit_off,
         if (unit_page_off[u + 1] <= unit_page_off[u]) continue;
         for (int i = 0; i < unit_len[u]; ++i) {
             int p = unit_target_pos[u] + i;
-            size_t slot = (size_t)unit_pages[unit_page_off[u] + i / page_size] * page_size + i % page_size;
-            int delta = p - (unit_cached_pos[u] + unit_cached_stride[u] * i);
+            int si = i + (unit_src_offset ? unit_src_offset[u] : 0);
+            size_t slot = (size_t)unit_pages[unit_page_off[u] + si / page_size] * page_size + si % page_size;
+            int tstride = unit_target_stride ? unit_target_stride[u] : 1;
+            int delta = (unit_target_pos[u] + tstride * i) - (unit_cached_pos[u] + unit_cached_stride[u] * i);
             delta_out[p] = delta;
             memcpy(v_asm + (size_t)p * row, v_pool + slot * row, row * sizeof(uint16_t));
             for (int h = 0; h < H_kv; ++h) {

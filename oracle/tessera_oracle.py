@@ -49,6 +49,11 @@ def _i32(a) -> np.ndarray:
     return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
 
 
+def _opt(w, name):
+    v = getattr(w, name, None)
+    return None if v is None else _i32(v)
+
+
 def bits(t) -> np.ndarray:
     """bf16 torch tensor (any device) -> contiguous uint16 numpy array of its bits."""
     import torch
@@ -78,7 +83,7 @@ def placement(w):
         ctypes.c_int(batch), _p(_i32(w.seq_len)), _p(_i32(w.unit_off)), _p(_i32(w.unit_len)),
         _p(_i32(w.unit_target_pos)), _p(_i32(w.unit_page_off)), _p(_i32(w.unit_pages)),
         _p(_i32(w.recompute_off)), _p(_i32(w.recompute_pos)), _p(_i32(w.free_pages)),
-        ctypes.c_int(len(w.free_pages)), ctypes.c_int(B),
+        ctypes.c_int(len(w.free_pages)), ctypes.c_int(B), _p(_opt(w, "unit_src_offset")),
         _p(page_off), _p(pages), _p(src_slot), _p(fresh))
     return st, page_off, pages[:n_pages], src_slot[:total], fresh[:total]
 
@@ -120,6 +125,7 @@ def assemble(w, r: int, k_pool_bits, v_pool_bits, k_new_bits, v_new_bits,
         ctypes.c_int(sh.head_dim), ctypes.c_double(sh.rope_theta), _p(inv_freq),
         ctypes.c_int(sh.rope_pairing),
         _p(k_pool_bits), _p(v_pool_bits), _p(k_new_bits), _p(v_new_bits),
+        _p(_opt(w, "unit_src_offset")), _p(_opt(w, "unit_target_stride")),
         _p(a.k), _p(a.v_bits), _p(a.k_bits), _p(a.k_exact), _p(a.delta))
     if st != 0:
         raise ValueError("oracle_assemble: request %d has positions nobody supplies" % r)

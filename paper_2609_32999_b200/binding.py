@@ -41,7 +41,8 @@ class ComposeDesc(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("seq_len", _I32P), ("unit_off", _I32P), ("unit_len", _I32P),
                 ("unit_cached_pos", _I32P), ("unit_cached_stride", _I32P), ("unit_target_pos", _I32P),
                 ("unit_page_off", _I32P), ("unit_pages", _I32P), ("recompute_off", _I32P),
-                ("recompute_pos", _I32P), ("free_pages", _I32P), ("n_free", ctypes.c_int32)]
+                ("recompute_pos", _I32P), ("free_pages", _I32P), ("n_free", ctypes.c_int32),
+                ("unit_src_offset", _I32P), ("unit_target_stride", _I32P)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -133,7 +134,11 @@ class Plan:
         cfg = ModelCfg(sh.num_q_heads, sh.num_kv_heads, sh.head_dim, sh.page_size, float(sh.rope_theta),
                        None if self._inv is None else self._inv.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
                        int(sh.rope_pairing), float(sh.sm_scale))
-        desc = ComposeDesc(len(a[0]), *[_ptr(x) for x in a], len(a[10]))
+        opt = [None if getattr(w, f, None) is None else _arr(getattr(w, f))
+               for f in ("unit_src_offset", "unit_target_stride")]
+        desc = ComposeDesc(len(a[0]), *[_ptr(x) for x in a[:11]], len(a[10]),
+                           *[None if x is None else _ptr(x) for x in opt])
+        self._opt = opt
         self._h = _vp()
         self.host_only = host_only
         st = _lib.tessera_plan_create(ctypes.byref(cfg), ctypes.byref(desc), int(w.num_pool_pages),

@@ -67,8 +67,10 @@ gather_rope_kernel(uint4 *__restrict__ k_pool, uint4 *__restrict__ v_pool,
 
     const GatherItem it = items[blockIdx.x];
     const int tid = threadIdx.x;
+    // rows row0, row0 + step, ... of the table; with step = -1 they are staged in ascending order
     const int n_rows = ROTATE ? (it.row_step ? it.count : 1) : 0;
-    for (int i = tid; i < n_rows * (D / 2); i += kThreads) s_rope[i] = rope[(size_t)it.row0 * (D / 2) + i];
+    const int first_row = it.row_step < 0 ? it.row0 - (it.count - 1) : it.row0;
+    for (int i = tid; i < n_rows * (D / 2); i += kThreads) s_rope[i] = rope[(size_t)first_row * (D / 2) + i];
     if (tid < it.count) {
         s_dst[tid] = g_dst[it.begin + tid];
         s_src[tid] = IN_PLACE ? s_dst[tid] : g_src[it.begin + tid];
@@ -122,7 +124,8 @@ gather_rope_kernel(uint4 *__restrict__ k_pool, uint4 *__restrict__ v_pool,
             }
             if (ROTATE) {
                 if (it.row_step != 0) {
-                    const float2 *row = s_rope + (size_t)tok[u] * (D / 2) + c * 8;
+                    const int sr = it.row_step < 0 ? it.count - 1 - tok[u] : tok[u];
+                    const float2 *row = s_rope + (size_t)sr * (D / 2) + c * 8;
                     float2 cr[8];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) cr[i] = row[i];

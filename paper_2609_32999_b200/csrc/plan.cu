@@ -77,8 +77,12 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
             if (d->unit_len[u] < 0) return fail(TESSERA_INVALID_ARG, fmt("unit %ld: negative length", u));
             int np = d->unit_page_off[u + 1] - d->unit_page_off[u];
             if (np < 0) return fail(TESSERA_INVALID_ARG, fmt("unit %ld: unit_page_off decreases", u));
-            if (np != 0 && np != (d->unit_len[u] + B - 1) / B)
+            const int off = d->unit_src_offset ? d->unit_src_offset[u] : 0;
+            if (off < 0 || off >= B) return fail(TESSERA_INVALID_ARG, fmt("unit %ld: source offset %ld outside [0, page_size)", u, off));
+            if (np != 0 && np != (off + d->unit_len[u] + B - 1) / B)
                 return fail(TESSERA_INVALID_ARG, fmt("unit %ld: %ld source pages for %ld tokens", u, np, d->unit_len[u]));
+            if (d->unit_target_stride && d->unit_target_stride[u] != 0 && d->unit_target_stride[u] != 1)
+                return fail(TESSERA_INVALID_ARG, fmt("unit %ld: target stride must be 0 or 1", u));
             if (np != 0 && d->unit_cached_stride[u] != 0 && d->unit_cached_stride[u] != 1)
                 return fail(TESSERA_INVALID_ARG, fmt("unit %ld: cached stride must be 0 or 1", u));
         }
@@ -141,8 +145,10 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
                 if (unit_of[base + tp + i] != -1)
                     return fail(TESSERA_UNIT_OVERLAP, fmt("units %ld and %ld both claim position %ld", unit_of[base + tp + i], u, tp + i));
                 unit_of[base + tp + i] = u;
-                if (cached)
-                    pl->src_slot[base + tp + i] = d->unit_pages[d->unit_page_off[u] + i / B] * B + i % B;
+                if (cached) {
+                    const int si = i + (d->unit_src_offset ? d->unit_src_offset[u] : 0);
+                    pl->src_slot[base + tp + i] = d->unit_pages[d->unit_page_off[u] + si / B] * B + si % B;
+                }
             }
         }
         for (int j = d->recompute_off[r]; j < d->recompute_off[r + 1]; ++j) {
@@ -164,9 +170,11 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
     for (int r = 0; r < batch; ++r)
         for (int u = d->unit_off[r]; u < d->unit_off[r + 1]; ++u) {
             if (d->unit_page_off[u + 1] <= d->unit_page_off[u]) continue;
+            // token i is shifted by (target_pos + ts * i) - (cached_pos + cs * i)
             const int64_t d0 = (int64_t)d->unit_target_pos[u] - d->unit_cached_pos[u];
-            if (d->unit_cached_stride[u] == 1) deltas.push_back(d0);
-            else for (int i = 0; i < d->unit_len[u]; ++i) deltas.push_back(d0 + i);
+            const int step = (d->unit_target_stride ? d->unit_target_stride[u] : 1) - d->unit_cached_stride[u];
+            if (step == 0) deltas.push_back(d0);
+            else for (int i = 0; i < d->unit_len[u]; ++i) deltas.push_back(d0 + (int64_t)step * i);
         }
     std::sort(deltas.begin(), deltas.end());
     deltas.erase(std::unique(deltas.begin(), deltas.end()), deltas.end());
@@ -190,8 +198,8 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
             if (d->unit_page_off[u + 1] <= d->unit_page_off[u]) continue;
             const int len = d->unit_len[u], tp = d->unit_target_pos[u];
             const int64_t d0 = (int64_t)tp - d->unit_cached_pos[u];
-            const int step = d->unit_cached_stride[u] == 1 ? 0 : 1;
-            const int32_t row0 = row_of(d0);       // stride 0: consecutive integers are consecutive rows
+            const int step = (d->unit_target_stride ? d->unit_target_stride[u] : 1) - d->unit_cached_stride[u];
+            const int32_t row0 = row_of(d0);       // step +-1: consecutive integers are consecutive rows
             for (int i0 = 0; i0 < len; i0 += kGatherItemTokens) {
                 const int cnt = std::min(kGatherItemTokens, len - i0);
                 pl->items.push_back({(int32_t)pl->g_src.size(), cnt, row0 + i0 * step, step});

@@ -52,6 +52,8 @@ class Workload:
     free_pages: np.ndarray          # destination page ids, consumed in order
     num_pool_pages: int
     n_layers: int = 1
+    unit_src_offset: Optional[np.ndarray] = None     # [n_units] token 0's offset inside its first source page
+    unit_target_stride: Optional[np.ndarray] = None  # [n_units] 0 = every token rotated for target_pos
 
     @property
     def batch(self) -> int:

@@ -152,3 +152,61 @@ def test_full_size_sampled(idx, n_random):
     tile_tokens = 128 // (w.shape.num_q_heads // w.shape.num_kv_heads)
     rows = {r: gu.sample_rows(w, r, rng, n_random // len(list(reqs)), tile_tokens) for r in reqs}
     gu.check_attention(g, asm, rows_by_request=rows)
+
+
+def _retention_workloads():
+    """A: a request with an uncached unit U at an unaligned position.  R: the plan that retains U from
+    A's pages into fresh cache pages in un-rotated form.  B: a later request that reuses the retained U
+    (cached without rotation) at another position."""
+    shape = wl.ModelShape(32, 8, 128, 64, 500000.0)
+    rng = np.random.default_rng(17)
+    pos_u, len_u = 37 + 200, 150
+    A = wl.build_workload("A", shape, [[37, wl.unit(200, "x", recompute=(0, 1)), wl.unit(len_u, "U", cached=False), 9]],
+                          rng, spare_pages=40)
+    B_ = shape.page_size
+    used = -(-int(A.seq_len[0]) // B_)
+    spare = A.free_pages[used:]
+    first, last = pos_u // B_, (pos_u + len_u - 1) // B_
+    n_cache = -(-len_u // B_)
+    i32 = lambda x: np.asarray(x, np.int32)
+    R = wl.Workload(name="retain", shape=shape, seq_len=i32([len_u]), unit_off=i32([0, 1]), unit_len=i32([len_u]),
+                    unit_cached_pos=i32([pos_u]), unit_cached_stride=i32([1]), unit_target_pos=i32([0]),
+                    unit_page_off=i32([0, last - first + 1]), unit_pages=i32(A.free_pages[first:last + 1]),
+                    recompute_off=i32([0, 0]), recompute_pos=i32([]), free_pages=i32(spare[:n_cache]),
+                    num_pool_pages=A.num_pool_pages, unit_src_offset=i32([pos_u % B_]), unit_target_stride=i32([0]))
+    tgt = 11
+    T_b = tgt + len_u + 5
+    B = wl.Workload(name="reuse", shape=shape, seq_len=i32([T_b]), unit_off=i32([0, 1]), unit_len=i32([len_u]),
+                    unit_cached_pos=i32([0]), unit_cached_stride=i32([0]), unit_target_pos=i32([tgt]),
+                    unit_page_off=i32([0, n_cache]), unit_pages=i32(spare[:n_cache]),
+                    recompute_off=i32([0, tgt + 5 + 2]),
+                    recompute_pos=i32(list(range(tgt)) + [tgt, tgt + 1] + list(range(tgt + len_u, T_b))),
+                    free_pages=i32(spare[n_cache:n_cache + -(-T_b // B_)]), num_pool_pages=A.num_pool_pages)
+    return A, R, B
+
+
+def test_retain_fresh_unit_then_reuse_it():
+    """Store side of the cache: a freshly computed unit is written back un-rotated from the request's
+    pages (source offset inside a page, shift = -(position) per token), then reused elsewhere."""
+    A, R, B = _retention_workloads()
+    a = gu.run_layer(A, seed=31)
+    assert a.status == 0
+    asm_a, _, _ = gu.check_assembled(a)
+    # retain: same pools, no poison (the sources are A's destination pages)
+    r = gu.run_layer(R, t=a.t, poison=False, attention=False)
+    gu.check_placement(r)
+    asm_r, kmx, kmean = gu.check_assembled(r)
+    gu.check_untouched(r)
+    assert set(asm_r[0].delta.tolist()) == set(range(-(237 + 149), -236))
+    # the retained keys are the fresh keys un-rotated: compare with the oracle applied to k_new of A
+    j0 = int(np.searchsorted(A.recompute_pos, 237))
+    fresh = orc.bf16_bits_to_f64(a.kn_bits[j0:j0 + 150])
+    for i in (0, 63, 149):
+        want = np.stack([orc.rope_rotate(fresh[i, h], -(237 + i), 500000.0) for h in range(8)])
+        assert np.max(np.abs(want - asm_r[0].k[i])) < 1e-9
+    # reuse the retained unit in another prompt
+    b = gu.run_layer(B, t=a.t, poison=False)
+    assert b.status == 0
+    gu.check_placement(b)
+    asm_b, _, _ = gu.check_assembled(b)
+    gu.check_attention(b, asm_b)

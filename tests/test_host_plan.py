@@ -106,3 +106,34 @@ def test_empty_batch_and_empty_request():
     plan = tb.Plan(w, host_only=True)
     page_off, pages, src = plan.block_table()
     assert list(page_off) == [0, 0, 1] and list(src) == [-1, -1, -1]
+
+
+def test_source_offset_and_target_stride_in_host_plan():
+    """Units read from the middle of a page (retention) and written without rotation."""
+    shape = wl.ModelShape(4, 2, 64, 16, 1e4)
+    i32 = lambda x: np.asarray(x, np.int32)
+    w = wl.Workload(name="retain", shape=shape, seq_len=i32([40]), unit_off=i32([0, 1]), unit_len=i32([40]),
+                    unit_cached_pos=i32([21]), unit_cached_stride=i32([1]), unit_target_pos=i32([0]),
+                    unit_page_off=i32([0, 3]), unit_pages=i32([7, 3, 9]), recompute_off=i32([0, 0]),
+                    recompute_pos=i32([]), free_pages=i32([12, 11, 10]), num_pool_pages=16,
+                    unit_src_offset=i32([5]), unit_target_stride=i32([0]))
+    plan = tb.Plan(w, host_only=True)
+    page_off, pages, src = plan.block_table()
+    st, o_off, o_pages, o_src, _ = orc.placement(w)
+    assert st == 0 and np.array_equal(src, o_src) and np.array_equal(pages, o_pages)
+    want = [[7, 3, 9][(5 + i) // 16] * 16 + (5 + i) % 16 for i in range(40)]
+    assert src.tolist() == want
+    assert plan.info.n_rope_rows == 40                      # one shift per token: -(21 + i)
+    # un-rotated form in the oracle: delta = -(cached_pos + i)
+    t = wl.make_tensors(w)
+    a = orc.assemble(w, 0, orc.bits(t.k_pool), orc.bits(t.v_pool), orc.bits(t.k_new), orc.bits(t.v_new))
+    assert a.delta.tolist() == [-(21 + i) for i in range(40)]
+    # wrong page count for the offset, bad offset, bad stride
+    ok = copy.deepcopy(w); ok.unit_src_offset = i32([0])                    # 40 tokens from 0 also span 3 pages
+    assert tb.plan_create_status(ok) == tb.OK
+    bad = copy.deepcopy(w); bad.unit_src_offset = i32([12])                 # 12 + 40 = 52 tokens need 4 pages, 3 given
+    assert tb.plan_create_status(bad) == tb.INVALID_ARG
+    bad = copy.deepcopy(w); bad.unit_src_offset = i32([16])
+    assert tb.plan_create_status(bad) == tb.INVALID_ARG
+    bad = copy.deepcopy(w); bad.unit_target_stride = i32([2])
+    assert tb.plan_create_status(bad) == tb.INVALID_ARG
