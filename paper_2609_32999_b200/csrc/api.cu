@@ -55,6 +55,7 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     const size_t o_pages = place<int32_t>(off, pl->pages.size());
     const size_t o_tiles = place<AttnTile>(off, pl->tiles.size());
     const size_t o_work = place<AttnWork>(off, pl->work.size());
+    const size_t o_workc = place<AttnWork>(off, pl->work_chunked.size());
     const size_t o_seq = place<int32_t>(off, pl->seq_len.size());
     const size_t o_status = place<int32_t>(off, 4);
     pl->host_blob.assign(off, 0);
@@ -71,6 +72,7 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     put(o_pages, pl->pages.data(), pl->pages.size() * 4);
     put(o_tiles, pl->tiles.data(), pl->tiles.size() * sizeof(AttnTile));
     put(o_work, pl->work.data(), pl->work.size() * sizeof(AttnWork));
+    put(o_workc, pl->work_chunked.data(), pl->work_chunked.size() * sizeof(AttnWork));
     put(o_seq, pl->seq_len.data(), pl->seq_len.size() * 4);
     TS_CUDA(cudaMalloc(&d.blob, off));
     TS_CUDA(cudaMemcpyAsync(d.blob, hb, off, cudaMemcpyHostToDevice, st));
@@ -86,6 +88,7 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     d.pages = reinterpret_cast<int32_t *>(db + o_pages);
     d.tiles = reinterpret_cast<AttnTile *>(db + o_tiles);
     d.work = reinterpret_cast<AttnWork *>(db + o_work);
+    d.work_chunked = reinterpret_cast<AttnWork *>(db + o_workc);
     d.seq_len = reinterpret_cast<int32_t *>(db + o_seq);
     d.status = reinterpret_cast<int32_t *>(db + o_status);
     return TESSERA_OK;
@@ -99,15 +102,33 @@ int32_t check_device_plan(const tessera_plan *pl) {
 
 bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
 
+// Fresh-row scatter + attention of the whole batch (chunk < 0) or of one request chunk.
 int32_t attention(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, const void *k_new,
-                  const void *v_new, void *out, float *lse, cudaStream_t st) {
-    TS_CUDA(launch_scatter_fresh(pl, k_pool, v_pool, k_new, v_new, st));
+                  const void *v_new, void *out, float *lse, int chunk, cudaStream_t st) {
+    TS_CUDA(launch_scatter_fresh(pl, k_pool, v_pool, k_new, v_new, chunk, st));
     if (pl->attn_kernel == 1) {
         std::string err;
-        cudaError_t e = launch_attn_tc(pl, k_pool, v_pool, q, out, lse, st, &err);
+        cudaError_t e = launch_attn_tc(pl, k_pool, v_pool, q, out, lse, chunk, st, &err);
         if (e != cudaSuccess) return set_error(TESSERA_CUDA_ERROR, "tcgen05 attention launch: " + err + " / " + cudaGetErrorString(e));
     } else {
-        TS_CUDA(launch_attn_simt(pl, k_pool, v_pool, q, out, lse, st));
+        TS_CUDA(launch_attn_simt(pl, k_pool, v_pool, q, out, lse, chunk, st));
+    }
+    return TESSERA_OK;
+}
+
+// Streams and events of the host-buffer entry point, created once per plan.
+int32_t ensure_pipeline(tessera_plan *pl) {
+    if (pl->s_in) return TESSERA_OK;
+    const size_t n = pl->chunk_row_off.size() - 1;
+    TS_CUDA(cudaStreamCreateWithFlags(&pl->s_in, cudaStreamNonBlocking));
+    TS_CUDA(cudaStreamCreateWithFlags(&pl->s_out, cudaStreamNonBlocking));
+    TS_CUDA(cudaEventCreateWithFlags(&pl->ev_start, cudaEventDisableTiming));
+    TS_CUDA(cudaEventCreateWithFlags(&pl->ev_out, cudaEventDisableTiming));
+    pl->ev_in.assign(n, nullptr);
+    pl->ev_comp.assign(n, nullptr);
+    for (size_t c = 0; c < n; ++c) {
+        TS_CUDA(cudaEventCreateWithFlags(&pl->ev_in[c], cudaEventDisableTiming));
+        TS_CUDA(cudaEventCreateWithFlags(&pl->ev_comp[c], cudaEventDisableTiming));
     }
     return TESSERA_OK;
 }
@@ -160,6 +181,12 @@ int32_t tessera_plan_destroy(tessera_plan *pl) {
     if (!pl) return TESSERA_OK;
     int32_t rc = TESSERA_OK;
     if (!pl->host_only) {
+        for (cudaEvent_t e : pl->ev_in) if (e) cudaEventDestroy(e);
+        for (cudaEvent_t e : pl->ev_comp) if (e) cudaEventDestroy(e);
+        if (pl->ev_start) cudaEventDestroy(pl->ev_start);
+        if (pl->ev_out) cudaEventDestroy(pl->ev_out);
+        if (pl->s_in) cudaStreamDestroy(pl->s_in);
+        if (pl->s_out) cudaStreamDestroy(pl->s_out);
         void *bufs[] = {pl->dev.blob, pl->dev.st_q, pl->dev.st_k, pl->dev.st_v, pl->dev.st_o, pl->dev.st_lse};
         for (void *b : bufs)
             if (b) {
@@ -233,7 +260,7 @@ int32_t tessera_partial_prefill_attn(const tessera_plan *pl, void *k_pool, void 
     if (pl->n_q > 0 && (!q || !out)) return set_error(TESSERA_INVALID_ARG, "q and out must be non-null");
     if (misaligned(q) || misaligned(out) || misaligned(k_new) || misaligned(v_new))
         return set_error(TESSERA_INVALID_ARG, "q / out / k_new / v_new must be 16-byte aligned");
-    return attention(pl, k_pool, v_pool, q, k_new, v_new, out, lse, static_cast<cudaStream_t>(stream));
+    return attention(pl, k_pool, v_pool, q, k_new, v_new, out, lse, -1, static_cast<cudaStream_t>(stream));
 }
 
 int32_t tessera_composed_prefill_host(tessera_plan *pl, void *k_pool, void *v_pool, const void *q_host,
@@ -255,18 +282,50 @@ int32_t tessera_composed_prefill_host(tessera_plan *pl, void *k_pool, void *v_po
         TS_CUDA(cudaMalloc(&d.st_v, kv_bytes));
         TS_CUDA(cudaMalloc(&d.st_o, q_bytes));
         TS_CUDA(cudaMalloc(reinterpret_cast<void **>(&d.st_lse), lse_bytes));
+        TS_CUDA(cudaMemsetAsync(d.st_q, 0, q_bytes, st));   // rows of later chunks are read (and discarded) as tile padding
     }
-    if (pl->n_q > 0) {
-        TS_CUDA(cudaMemcpyAsync(d.st_q, q_host, q_bytes, cudaMemcpyHostToDevice, st));
-        TS_CUDA(cudaMemcpyAsync(d.st_k, k_new_host, kv_bytes, cudaMemcpyHostToDevice, st));
-        TS_CUDA(cudaMemcpyAsync(d.st_v, v_new_host, kv_bytes, cudaMemcpyHostToDevice, st));
+    if (pl->n_q == 0) {
+        TS_CUDA(launch_gather(pl, k_pool, v_pool, GatherMode::kCopyRotate, st));
+        TS_CUDA(cudaStreamSynchronize(st));
+        return TESSERA_OK;
+    }
+    // Chunks of whole requests flow through three streams: host->device copies of chunk c+1, compute
+    // of chunk c and device->host copies of chunk c-1 overlap.  The gather needs no activations and
+    // runs while the first chunk is on its way.
+    if (int32_t rc = ensure_pipeline(pl)) return rc;
+    const size_t q_row = (size_t)pl->cfg.num_q_heads * pl->cfg.head_dim * 2;
+    const size_t kv_row = (size_t)pl->cfg.num_kv_heads * pl->cfg.head_dim * 2;
+    const size_t lse_row = (size_t)pl->cfg.num_q_heads * sizeof(float);
+    const int n_chunks = (int)pl->chunk_row_off.size() - 1;
+    auto at = [](const void *p, size_t off) { return static_cast<const char *>(p) + off; };
+    auto at_w = [](void *p, size_t off) { return static_cast<char *>(p) + off; };
+    TS_CUDA(cudaEventRecord(pl->ev_start, st));
+    TS_CUDA(cudaStreamWaitEvent(pl->s_in, pl->ev_start, 0));
+    TS_CUDA(cudaStreamWaitEvent(pl->s_out, pl->ev_start, 0));
+    for (int c = 0; c < n_chunks; ++c) {
+        const size_t r0 = pl->chunk_row_off[c], rows = pl->chunk_row_off[c + 1] - r0;
+        if (rows) {
+            TS_CUDA(cudaMemcpyAsync(at_w(d.st_q, r0 * q_row), at(q_host, r0 * q_row), rows * q_row, cudaMemcpyHostToDevice, pl->s_in));
+            TS_CUDA(cudaMemcpyAsync(at_w(d.st_k, r0 * kv_row), at(k_new_host, r0 * kv_row), rows * kv_row, cudaMemcpyHostToDevice, pl->s_in));
+            TS_CUDA(cudaMemcpyAsync(at_w(d.st_v, r0 * kv_row), at(v_new_host, r0 * kv_row), rows * kv_row, cudaMemcpyHostToDevice, pl->s_in));
+        }
+        TS_CUDA(cudaEventRecord(pl->ev_in[c], pl->s_in));
     }
     TS_CUDA(launch_gather(pl, k_pool, v_pool, GatherMode::kCopyRotate, st));
-    if (int32_t rc = attention(pl, k_pool, v_pool, d.st_q, d.st_k, d.st_v, d.st_o, d.st_lse, st)) return rc;
-    if (pl->n_q > 0) {
-        TS_CUDA(cudaMemcpyAsync(out_host, d.st_o, q_bytes, cudaMemcpyDeviceToHost, st));
-        if (lse_host) TS_CUDA(cudaMemcpyAsync(lse_host, d.st_lse, lse_bytes, cudaMemcpyDeviceToHost, st));
+    for (int c = 0; c < n_chunks; ++c) {
+        const size_t r0 = pl->chunk_row_off[c], rows = pl->chunk_row_off[c + 1] - r0;
+        TS_CUDA(cudaStreamWaitEvent(st, pl->ev_in[c], 0));
+        if (int32_t rc = attention(pl, k_pool, v_pool, d.st_q, d.st_k, d.st_v, d.st_o, d.st_lse, c, st)) return rc;
+        TS_CUDA(cudaEventRecord(pl->ev_comp[c], st));
+        TS_CUDA(cudaStreamWaitEvent(pl->s_out, pl->ev_comp[c], 0));
+        if (rows) {
+            TS_CUDA(cudaMemcpyAsync(at_w(out_host, r0 * q_row), at(d.st_o, r0 * q_row), rows * q_row, cudaMemcpyDeviceToHost, pl->s_out));
+            if (lse_host)
+                TS_CUDA(cudaMemcpyAsync(at_w(lse_host, r0 * lse_row), at(d.st_lse, r0 * lse_row), rows * lse_row, cudaMemcpyDeviceToHost, pl->s_out));
+        }
     }
+    TS_CUDA(cudaEventRecord(pl->ev_out, pl->s_out));
+    TS_CUDA(cudaStreamWaitEvent(st, pl->ev_out, 0));
     TS_CUDA(cudaStreamSynchronize(st));
     return TESSERA_OK;
 }

@@ -16,10 +16,10 @@ __global__ void attn_simt_kernel(const __nv_bfloat16 *__restrict__ k_pool, const
                                  float *__restrict__ lse, const int32_t *__restrict__ q_pos,
                                  const int32_t *__restrict__ q_req, const int32_t *__restrict__ page_off,
                                  const int32_t *__restrict__ pages, int H_q, int H_kv, int page_size,
-                                 float scale_log2) {
+                                 float scale_log2, int row0) {
     constexpr int EPL = D / 32;                      // output elements per lane
     extern __shared__ float s_q[];                   // [g][D]
-    const int j = blockIdx.x, kvh = blockIdx.y;
+    const int j = row0 + blockIdx.x, kvh = blockIdx.y;
     const int g = H_q / H_kv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = kvh * g + warp;
@@ -98,11 +98,14 @@ __global__ void attn_simt_kernel(const __nv_bfloat16 *__restrict__ k_pool, const
 }  // namespace
 
 cudaError_t launch_attn_simt(const tessera_plan *pl, const void *k_pool, const void *v_pool, const void *q,
-                             void *out, float *lse, cudaStream_t st) {
+                             void *out, float *lse, int chunk, cudaStream_t st) {
     if (pl->n_q == 0) return cudaSuccess;
+    const int row0 = chunk < 0 ? 0 : pl->chunk_row_off[chunk];
+    const int64_t rows = chunk < 0 ? pl->n_q : pl->chunk_row_off[chunk + 1] - row0;
+    if (rows == 0) return cudaSuccess;
     const int Hq = pl->cfg.num_q_heads, Hkv = pl->cfg.num_kv_heads, D = pl->cfg.head_dim, g = Hq / Hkv;
     const float scale_log2 = pl->sm_scale * 1.4426950408889634f;
-    dim3 grid((unsigned)pl->n_q, (unsigned)Hkv);
+    dim3 grid((unsigned)rows, (unsigned)Hkv);
     const DeviceTables &d = pl->dev;
     auto *kp = static_cast<const __nv_bfloat16 *>(k_pool);
     auto *vp = static_cast<const __nv_bfloat16 *>(v_pool);
@@ -110,9 +113,9 @@ cudaError_t launch_attn_simt(const tessera_plan *pl, const void *k_pool, const v
     auto *op = static_cast<__nv_bfloat16 *>(out);
     const size_t smem = (size_t)g * D * sizeof(float);
     if (D == 128)
-        attn_simt_kernel<128><<<grid, g * 32, smem, st>>>(kp, vp, qp, op, lse, d.q_pos, d.q_req, d.page_off, d.pages, Hq, Hkv, pl->cfg.page_size, scale_log2);
+        attn_simt_kernel<128><<<grid, g * 32, smem, st>>>(kp, vp, qp, op, lse, d.q_pos, d.q_req, d.page_off, d.pages, Hq, Hkv, pl->cfg.page_size, scale_log2, row0);
     else
-        attn_simt_kernel<64><<<grid, g * 32, smem, st>>>(kp, vp, qp, op, lse, d.q_pos, d.q_req, d.page_off, d.pages, Hq, Hkv, pl->cfg.page_size, scale_log2);
+        attn_simt_kernel<64><<<grid, g * 32, smem, st>>>(kp, vp, qp, op, lse, d.q_pos, d.q_req, d.page_off, d.pages, Hq, Hkv, pl->cfg.page_size, scale_log2, row0);
     count_launch();
     return cudaGetLastError();
 }

@@ -474,8 +474,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 }  // namespace
 
 cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
-                           float *lse, cudaStream_t st, std::string *err) {
+                           float *lse, int chunk, cudaStream_t st, std::string *err) {
     if (pl->n_q == 0 || pl->work.empty()) return cudaSuccess;
+    const AttnWork *work = chunk < 0 ? pl->dev.work : pl->dev.work_chunked + pl->chunk_work_off[chunk];
+    const size_t n_work = chunk < 0 ? pl->work.size() : (size_t)(pl->chunk_work_off[chunk + 1] - pl->chunk_work_off[chunk]);
+    if (n_work == 0) return cudaSuccess;
     const int Hq = pl->cfg.num_q_heads, Hkv = pl->cfg.num_kv_heads, g = Hq / Hkv;
     if (pl->cfg.head_dim != kD || pl->cfg.page_size != kPage || kRows % g != 0) {
         *err = "shape outside the tcgen05 kernel's range";
@@ -491,8 +494,8 @@ cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, c
     }
     const DeviceTables &d = pl->dev;
     const float scale_log2 = pl->sm_scale * 1.4426950408889634f;
-    attn_tc_kernel<<<(unsigned)pl->work.size(), kThreads, kSmemAlloc, st>>>(
-        tq, tk, tv, d.tiles, d.work, d.q_pos, d.page_off, d.pages, d.seq_len,
+    attn_tc_kernel<<<(unsigned)n_work, kThreads, kSmemAlloc, st>>>(
+        tq, tk, tv, d.tiles, work, d.q_pos, d.page_off, d.pages, d.seq_len,
         static_cast<__nv_bfloat16 *>(out), lse, Hq, g, pl->num_pool_pages, scale_log2, d.status);
     count_launch();
     cudaError_t e = cudaGetLastError();

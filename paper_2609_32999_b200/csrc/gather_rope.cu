@@ -145,8 +145,9 @@ gather_rope_kernel(uint4 *__restrict__ k_pool, uint4 *__restrict__ v_pool,
 __global__ void __launch_bounds__(256)
 scatter_fresh_kernel(uint4 *__restrict__ k_pool, uint4 *__restrict__ v_pool,
                      const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
-                     const int32_t *__restrict__ fresh_dst, int64_t n_chunks, int row_chunks) {
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_chunks; e += (int64_t)gridDim.x * blockDim.x) {
+                     const int32_t *__restrict__ fresh_dst, int64_t first_chunk, int64_t n_chunks, int row_chunks) {
+    for (int64_t e = first_chunk + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < first_chunk + n_chunks;
+         e += (int64_t)gridDim.x * blockDim.x) {
         const int64_t j = e / row_chunks;
         const int c = (int)(e - j * row_chunks);
         const size_t o = (size_t)fresh_dst[j] * row_chunks + c;
@@ -186,14 +187,17 @@ cudaError_t launch_gather(const tessera_plan *pl, void *k_pool, void *v_pool, Ga
 }
 
 cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_pool, const void *k_new,
-                                 const void *v_new, cudaStream_t st) {
+                                 const void *v_new, int chunk, cudaStream_t st) {
     if (pl->n_q == 0 || (!k_new && !v_new)) return cudaSuccess;
     const int row_chunks = pl->cfg.num_kv_heads * pl->cfg.head_dim / 8;
-    const int64_t n_chunks = pl->n_q * row_chunks;
+    const int64_t row0 = chunk < 0 ? 0 : pl->chunk_row_off[chunk];
+    const int64_t rows = chunk < 0 ? pl->n_q : pl->chunk_row_off[chunk + 1] - row0;
+    if (rows == 0) return cudaSuccess;
+    const int64_t n_chunks = rows * row_chunks;
     const int blocks = (int)std::min<int64_t>((n_chunks + 255) / 256, 148 * 16);
     scatter_fresh_kernel<<<blocks, 256, 0, st>>>(static_cast<uint4 *>(k_pool), static_cast<uint4 *>(v_pool),
                                                 static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new),
-                                                pl->dev.fresh_dst, n_chunks, row_chunks);
+                                                pl->dev.fresh_dst, row0 * row_chunks, n_chunks, row_chunks);
     count_launch();
     return cudaGetLastError();
 }

@@ -11,12 +11,14 @@ enum class GatherMode { kCopy, kCopyRotate, kShiftInPlace };
 void count_launch();   // bumps the process-wide kernel-launch counter
 
 cudaError_t launch_gather(const tessera_plan *pl, void *k_pool, void *v_pool, GatherMode mode, cudaStream_t st);
+// chunk < 0: the whole batch; otherwise only request chunk `chunk` (see tessera_plan::chunk_row_off).
+// k_new / v_new / q / out / lse always point at row 0 of the whole batch.
 cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_pool, const void *k_new,
-                                 const void *v_new, cudaStream_t st);
+                                 const void *v_new, int chunk, cudaStream_t st);
 cudaError_t launch_attn_simt(const tessera_plan *pl, const void *k_pool, const void *v_pool, const void *q,
-                             void *out, float *lse, cudaStream_t st);
+                             void *out, float *lse, int chunk, cudaStream_t st);
 // tcgen05 path; returns cudaErrorNotSupported when the plan's shape is outside its range.
 cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
-                           float *lse, cudaStream_t st, std::string *err);
+                           float *lse, int chunk, cudaStream_t st, std::string *err);
 
 }  // namespace tessera

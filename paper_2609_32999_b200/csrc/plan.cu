@@ -248,16 +248,57 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
             if (w.tile_b >= 0) c += (pl->tiles[w.tile_b].kv_len + page - 1) / page;
             return c;
         };
+        auto sort_items = [&](std::vector<AttnWork>::iterator first_it, std::vector<AttnWork>::iterator last_it) {
+            int max_cost = 1;
+            for (auto it = first_it; it != last_it; ++it) max_cost = std::max(max_cost, cost(*it));
+            const int band = std::max(1, max_cost / kAttnCostBands);
+            auto key = [&](const AttnWork &w) {
+                return std::make_tuple(-(cost(w) / band), pl->tiles[w.tile_a].req, w.kvh, -cost(w));
+            };
+            std::stable_sort(first_it, last_it, [&](const AttnWork &x, const AttnWork &y) { return key(x) < key(y); });
+        };
+        // chunks of whole requests with about equal attention cost, for the host-buffer pipeline
+        std::vector<int64_t> req_cost(batch, 0);
+        for (const AttnWork &w : pl->work) req_cost[pl->tiles[w.tile_a].req] += cost(w);
+        if (pl->attn_kernel != 1)      // generic kernel: cost = (query, key) pairs of the request
+            for (int r = 0; r < batch; ++r) {
+                req_cost[r] = 0;
+                for (int j = d->recompute_off[r]; j < d->recompute_off[r + 1]; ++j) req_cost[r] += d->recompute_pos[j] + 1;
+            }
+        int64_t total_cost = 0;
+        for (int64_t c : req_cost) total_cost += c;
+        const int n_chunks = std::max(1, std::min(batch, kHostChunks));
+        std::vector<int> chunk_of(batch, 0);
+        pl->chunk_row_off.assign(1, 0);
+        {
+            int64_t acc = 0;
+            int c = 0;
+            for (int r = 0; r < batch; ++r) {
+                chunk_of[r] = c;
+                acc += req_cost[r];
+                const bool last_req = r + 1 == batch;
+                // close the chunk when its share of the cost is reached, keeping one request per remaining chunk
+                if (!last_req && c + 1 < n_chunks && (acc * n_chunks >= total_cost * (c + 1) || batch - (r + 1) <= n_chunks - (c + 1))) {
+                    pl->chunk_row_off.push_back(d->recompute_off[r + 1]);
+                    ++c;
+                }
+            }
+            pl->chunk_row_off.push_back(n_q);
+        }
+        const int used_chunks = (int)pl->chunk_row_off.size() - 1;
+        pl->work_chunked = pl->work;
+        std::stable_sort(pl->work_chunked.begin(), pl->work_chunked.end(), [&](const AttnWork &x, const AttnWork &y) {
+            return chunk_of[pl->tiles[x.tile_a].req] < chunk_of[pl->tiles[y.tile_a].req];
+        });
+        pl->chunk_work_off.assign(used_chunks + 1, 0);
+        for (const AttnWork &w : pl->work_chunked) ++pl->chunk_work_off[chunk_of[pl->tiles[w.tile_a].req] + 1];
+        for (int c = 0; c < used_chunks; ++c) pl->chunk_work_off[c + 1] += pl->chunk_work_off[c];
+        for (int c = 0; c < used_chunks; ++c)
+            sort_items(pl->work_chunked.begin() + pl->chunk_work_off[c], pl->work_chunked.begin() + pl->chunk_work_off[c + 1]);
         // Longest first in coarse cost bands; inside a band, items of one (request, KV head) stay
         // together, so thread blocks that run at the same time stream the same K/V pages and find
         // them in L2.
-        int max_cost = 1;
-        for (const AttnWork &w : pl->work) max_cost = std::max(max_cost, cost(w));
-        const int band = std::max(1, max_cost / kAttnCostBands);
-        auto key = [&](const AttnWork &w) {
-            return std::make_tuple(-(cost(w) / band), pl->tiles[w.tile_a].req, w.kvh, -cost(w));
-        };
-        std::stable_sort(pl->work.begin(), pl->work.end(), [&](const AttnWork &x, const AttnWork &y) { return key(x) < key(y); });
+        sort_items(pl->work.begin(), pl->work.end());
     }
 
     pl->total_tokens = total;

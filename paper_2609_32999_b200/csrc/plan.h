@@ -4,6 +4,7 @@
 #include <string>
 #include <vector>
 
+#include <cuda_runtime.h>
 #include <vector_types.h>
 
 #include "tessera.h"
@@ -13,6 +14,7 @@ namespace tessera {
 constexpr int kGatherItemTokens = 32;   // token rows per thread block of the gather kernel
 constexpr int kAttnTileRows = 128;      // query rows (tokens x grouped heads) per tcgen05 tile
 constexpr bool kHaveTensorCoreKernel = true;
+constexpr int kHostChunks = 4;          // request chunks of the host-buffer entry point's copy / compute pipeline
 constexpr int kAttnCostBands = 16;      // cost bands of the attention work list (longest band first)
 
 // One thread block of the gather / shift kernel: `count` consecutive entries of the copy list that
@@ -45,6 +47,7 @@ struct DeviceTables {
     int32_t *pages = nullptr;      // block tables
     AttnTile *tiles = nullptr;
     AttnWork *work = nullptr;      // tcgen05 work items, longest first
+    AttnWork *work_chunked = nullptr;  // the same items grouped by request chunk (host-buffer entry)
     int32_t *seq_len = nullptr;    // [batch]
     int32_t *status = nullptr;     // device status word(s)
     // staging for the host-buffer entry point (allocated on first use)
@@ -71,6 +74,9 @@ struct tessera_plan {
     std::vector<float> rope_table;         // [rows][D/2][2]
     std::vector<tessera::AttnTile> tiles;
     std::vector<tessera::AttnWork> work;
+    // The host-buffer entry point pipelines copies against compute over chunks of whole requests.
+    std::vector<tessera::AttnWork> work_chunked;   // items of chunk c: [chunk_work_off[c], chunk_work_off[c+1])
+    std::vector<int32_t> chunk_work_off, chunk_row_off;   // [n_chunks + 1]; rows = recompute rows
     int32_t attn_kernel = 0;
     int32_t tile_tokens = 0;
 
@@ -78,6 +84,10 @@ struct tessera_plan {
 
     std::vector<char> host_blob;           // staging image of the device tables
     tessera::DeviceTables dev;
+    // streams / events of the host-buffer entry point (created on first use)
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_out = nullptr;
+    std::vector<cudaEvent_t> ev_in, ev_comp;
 };
 
 namespace tessera {
