@@ -56,9 +56,15 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     const size_t o_tiles = place<AttnTile>(off, pl->tiles.size());
     const size_t o_work = place<AttnWork>(off, pl->work.size());
     const size_t o_workc = place<AttnWork>(off, pl->work_chunked.size());
+    const size_t o_comb = place<CombineItem>(off, pl->combine.size());
     const size_t o_seq = place<int32_t>(off, pl->seq_len.size());
     const size_t o_status = place<int32_t>(off, 4);
-    pl->host_blob.assign(off, 0);
+    // split-KV workspace: one slot per (tile, KV head, part)
+    const size_t n_slots = pl->max_parts > 1 ? pl->tiles.size() * pl->cfg.num_kv_heads * pl->max_parts : 0;
+    const size_t o_wsml = place<float2>(off, n_slots * kAttnTileRows);
+    const size_t o_wso = place<float>(off, n_slots * kAttnTileRows * pl->cfg.head_dim);
+    const size_t table_bytes = o_wsml;    // the workspace behind it needs no upload
+    pl->host_blob.assign(table_bytes, 0);
     char *hb = pl->host_blob.data();
     auto put = [&](size_t o, const void *src, size_t bytes) { if (bytes) std::memcpy(hb + o, src, bytes); };
     put(o_src, pl->g_src.data(), pl->g_src.size() * 4);
@@ -73,9 +79,10 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     put(o_tiles, pl->tiles.data(), pl->tiles.size() * sizeof(AttnTile));
     put(o_work, pl->work.data(), pl->work.size() * sizeof(AttnWork));
     put(o_workc, pl->work_chunked.data(), pl->work_chunked.size() * sizeof(AttnWork));
+    put(o_comb, pl->combine.data(), pl->combine.size() * sizeof(CombineItem));
     put(o_seq, pl->seq_len.data(), pl->seq_len.size() * 4);
     TS_CUDA(cudaMalloc(&d.blob, off));
-    TS_CUDA(cudaMemcpyAsync(d.blob, hb, off, cudaMemcpyHostToDevice, st));
+    TS_CUDA(cudaMemcpyAsync(d.blob, hb, table_bytes, cudaMemcpyHostToDevice, st));
     char *db = static_cast<char *>(d.blob);
     d.g_src = reinterpret_cast<int32_t *>(db + o_src);
     d.g_dst = reinterpret_cast<int32_t *>(db + o_dst);
@@ -89,6 +96,9 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     d.tiles = reinterpret_cast<AttnTile *>(db + o_tiles);
     d.work = reinterpret_cast<AttnWork *>(db + o_work);
     d.work_chunked = reinterpret_cast<AttnWork *>(db + o_workc);
+    d.combine = reinterpret_cast<CombineItem *>(db + o_comb);
+    d.ws_ml = reinterpret_cast<float2 *>(db + o_wsml);
+    d.ws_o = reinterpret_cast<float *>(db + o_wso);
     d.seq_len = reinterpret_cast<int32_t *>(db + o_seq);
     d.status = reinterpret_cast<int32_t *>(db + o_status);
     return TESSERA_OK;

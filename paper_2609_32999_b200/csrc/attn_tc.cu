@@ -100,7 +100,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                const AttnWork *__restrict__ work, const int32_t *__restrict__ q_pos,
                const int32_t *__restrict__ page_off, const int32_t *__restrict__ pages,
                const int32_t *__restrict__ seq_len, __nv_bfloat16 *__restrict__ out, float *__restrict__ lse,
-               int H_q, int g, int num_pool_pages, float scale_log2, int *status) {
+               int H_q, int g, int H_kv, int num_pool_pages, float scale_log2, int max_parts,
+               float *__restrict__ ws_o, float2 *__restrict__ ws_ml, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     __shared__ __align__(8) Barriers bars;
@@ -127,8 +128,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const AttnTile t0 = tiles[wk.tile_a];
     const AttnTile t1 = tiles[n_tiles == 2 ? wk.tile_b : wk.tile_a];
     const int kvh = wk.kvh;
-    const int n_steps0 = (t0.kv_len + kStep - 1) / kStep;
-    const int n_steps1 = n_tiles == 2 ? (t1.kv_len + kStep - 1) / kStep : 0;
+    // This block covers the 128-key steps [step0, step_end) of its tiles (all of them unless the item
+    // was split); step indices below are relative to step0.
+    const int step0 = wk.step_begin;
+    const int n_steps0 = min(wk.step_end, (t0.kv_len + kStep - 1) / kStep) - step0;
+    const int n_steps1 = n_tiles == 2 ? min(wk.step_end, (t1.kv_len + kStep - 1) / kStep) - step0 : 0;
     const int n_steps = max(n_steps0, n_steps1);
     const int T = seq_len[t0.req];
     const int req_pages = (T + kPage - 1) / kPage;
@@ -182,7 +186,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int j0 = 0; j0 < n_steps; j0 += 16) {
             // lane l holds the id of page (2 * j0 + l); a page past the request's last one is fetched
             // from outside the pool, which TMA fills with zeros
-            const int pi = 2 * j0 + lane;
+            const int pi = 2 * (step0 + j0) + lane;
             const int my_page = pi < req_pages ? bt[pi] : num_pool_pages;
             const int jn = min(16, n_steps - j0);
             for (int jj = 0; jj < jn; ++jj) {
@@ -217,7 +221,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         constexpr uint32_t idesc_o = idesc_bf16(kRows, kD, true);
         const int q = warp - 9;
         const int my_steps = q ? n_steps1 : n_steps0;
-        const int tail_step = (T % kStep) ? T / kStep : -1;        // step holding slots past the sequence end
+        const int tail_step = (T % kStep) ? T / kStep - step0 : -1;   // step holding slots past the sequence end
         const uint32_t qbase = smem_u32(sm + kSmemQ + q * kQTileBytes);
         const uint32_t tS = tmem + kTmemS + q * 128, tO = tmem + kTmemO + q * 128;
 
@@ -261,7 +265,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 // probabilities are zero, but 0 x NaN would still poison the accumulator.  (Both
                 // issuing warps may write these zeros; the values agree.)
                 uint8_t *v = sm + kSmemRing + vslot * kSlotBytes;
-                for (int r = T - j * kStep; r < kStep; ++r)
+                for (int r = T - (step0 + j) * kStep; r < kStep; ++r)
                     if (lane < 16) *reinterpret_cast<uint4 *>(v + (lane >> 3) * kHalfBytes + r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
                 fence_proxy_async_smem();
                 __syncwarp();
@@ -320,8 +324,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 mbar_wait(smem_u32(&bars.s_full[q]), j & 1, abort_flag, status, 7);
                 tc_fence_after();
                 if (tid == 0) TRACE(q, j, 1);
-                const int key0 = j * kStep + h * 64;
-                const bool masked = j * kStep + kStep > (q ? t1.kv_full : t0.kv_full);   // a causal limit falls in this step
+                const int key0 = (step0 + j) * kStep + h * 64;
+                const bool masked = (step0 + j) * kStep + kStep > (q ? t1.kv_full : t0.kv_full);   // a causal limit falls in this step
                 const int pr = p_row[q];
 
                 uint32_t pk[32];
@@ -348,7 +352,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     }
                     if (with_exp) {
                         float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
-                        const float neg_m = -m_row[q];
+                        // a row that has seen no visible key yet (possible in a later split-KV part) keeps
+                        // the reference at 0: its scores are all -inf and its probabilities 0
+                        const float neg_m = m_row[q] == -INFINITY ? 0.f : -m_row[q];
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             float x0, x1;
@@ -383,8 +389,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     s_xchg[h][row] = mx;
                     named_sync(1 + pair, 64);
                     const float mc = fmaxf(m_row[q], fmaxf(mx, s_xchg[h ^ 1][row]) * scale_log2);
-                    factor = ex2(m_row[q] - mc);       // 0 on the first step (m_row = -inf)
-                    m_row[q] = mc;
+                    if (mc != -INFINITY) {
+                        factor = ex2(m_row[q] - mc);   // 0 when the row had no visible key before
+                        m_row[q] = mc;
+                    }
                     named_sync(1 + pair, 64);          // s_xchg may be rewritten after this point
                     if (j > 0) {
                         const uint32_t tO = tmem + kTmemO + q * 128 + h * 64 + lane_base;
@@ -423,6 +431,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int q = 0; q < n_tiles; ++q) {
             const AttnTile &t = q ? t1 : t0;
             const float l_tot = l_row[q] + l_xchg[(q * 2 + (h ^ 1)) * 128 + row];
+            if (wk.n_parts > 1) {
+                // split-KV part: unnormalised accumulator, reference maximum and sum go to the workspace
+                const size_t slot = ((size_t)(q ? wk.tile_b : wk.tile_a) * H_kv + kvh) * max_parts + wk.part;
+                float *po = ws_o + (slot * kRows + row) * kD + h * 64;
+                const uint32_t tOp = tmem + kTmemO + q * 128 + h * 64 + lane_base;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tOp + c * 32, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        *reinterpret_cast<uint4 *>(po + c * 32 + v * 4) = make_uint4(o[v * 4], o[v * 4 + 1], o[v * 4 + 2], o[v * 4 + 3]);
+                }
+                if (h == 0) ws_ml[slot * kRows + row] = make_float2(m_row[q], l_tot);
+                continue;
+            }
             const float inv = 1.f / l_tot;
             const int head = kvh * g + row % g;
             __nv_bfloat16 *orow = out + ((size_t)(t.q_begin + tok[q]) * H_q + head) * kD + h * 64;
@@ -471,6 +496,38 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     if (warp == 9) tmem_dealloc(tmem, kTmemCols);
 }
 
+// Merges the parts of a split-KV launch: for every row, O = sum_p O_p 2^(m_p - m) / sum_p l_p 2^(m_p - m)
+// with m = max_p m_p.  One block per (tile, KV head); a warp walks rows, lanes walk head_dim.
+__global__ void __launch_bounds__(256)
+attn_combine_kernel(const CombineItem *__restrict__ items, const AttnTile *__restrict__ tiles,
+                    const float *__restrict__ ws_o, const float2 *__restrict__ ws_ml, __nv_bfloat16 *__restrict__ out,
+                    float *__restrict__ lse, int H_q, int H_kv, int g, int max_parts) {
+    const CombineItem it = items[blockIdx.x];
+    const AttnTile t = tiles[it.tile];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const size_t slot0 = ((size_t)it.tile * H_kv + it.kvh) * max_parts;
+    for (int row = warp; row < t.n_tok * g; row += 8) {
+        float m = -INFINITY;
+        for (int p = 0; p < it.n_parts; ++p) m = fmaxf(m, ws_ml[(slot0 + p) * kRows + row].x);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float l = 0.f;
+        for (int p = 0; p < it.n_parts; ++p) {
+            const float2 ml = ws_ml[(slot0 + p) * kRows + row];
+            const float w = exp2f(ml.x - m);
+            l += ml.y * w;
+            const float4 o = *reinterpret_cast<const float4 *>(ws_o + ((slot0 + p) * kRows + row) * kD + lane * 4);
+            acc.x = fmaf(o.x, w, acc.x); acc.y = fmaf(o.y, w, acc.y); acc.z = fmaf(o.z, w, acc.z); acc.w = fmaf(o.w, w, acc.w);
+        }
+        const float inv = 1.f / l;
+        const int tok = t.q_begin + row / g, head = it.kvh * g + row % g;
+        uint2 pk;
+        pk.x = pack_bf16(acc.x * inv, acc.y * inv);
+        pk.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2 *>(out + ((size_t)tok * H_q + head) * kD + lane * 4) = pk;
+        if (lse && lane == 0) lse[(size_t)tok * H_q + head] = (m + log2f(l)) * 0.6931471805599453f;
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
@@ -496,8 +553,17 @@ cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, c
     const float scale_log2 = pl->sm_scale * 1.4426950408889634f;
     attn_tc_kernel<<<(unsigned)n_work, kThreads, kSmemAlloc, st>>>(
         tq, tk, tv, d.tiles, work, d.q_pos, d.page_off, d.pages, d.seq_len,
-        static_cast<__nv_bfloat16 *>(out), lse, Hq, g, pl->num_pool_pages, scale_log2, d.status);
+        static_cast<__nv_bfloat16 *>(out), lse, Hq, g, Hkv, pl->num_pool_pages, scale_log2, pl->max_parts, d.ws_o, d.ws_ml, d.status);
     count_launch();
+    if (pl->max_parts > 1) {
+        const int c0 = chunk < 0 ? 0 : pl->chunk_combine_off[chunk];
+        const int c1 = chunk < 0 ? (int)pl->combine.size() : pl->chunk_combine_off[chunk + 1];
+        if (c1 > c0) {
+            attn_combine_kernel<<<c1 - c0, 256, 0, st>>>(d.combine + c0, d.tiles, d.ws_o, d.ws_ml, static_cast<__nv_bfloat16 *>(out),
+                                                          lse, Hq, Hkv, g, pl->max_parts);
+            count_launch();
+        }
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) *err = "kernel launch";
     return e;

@@ -232,20 +232,56 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
     pl->work.clear();
     {
         const int page = 2 * B;      // the kernel advances two pages per step
+        std::vector<std::pair<int32_t, int32_t>> pairs;
         size_t first = 0;
         while (first < pl->tiles.size()) {
             size_t last = first;
             while (last < pl->tiles.size() && pl->tiles[last].req == pl->tiles[first].req) ++last;
             for (size_t k = first; k < last; k += 2) {
                 const int32_t a = (int32_t)k, b2 = (k + 1 < last) ? (int32_t)(k + 1) : -1;
-                const int steps = (pl->tiles[b2 >= 0 ? b2 : a].kv_len + page - 1) / page;
-                for (int h = 0; h < Hkv; ++h) pl->work.push_back({a, b2, h, steps});
+                pairs.push_back({a, b2});
             }
             first = last;
         }
+        auto steps_of = [&](int32_t tile) { return (pl->tiles[tile].kv_len + page - 1) / page; };
+        // Split-KV: a batch with fewer items than SMs (a single request, typically) splits each item's
+        // key range into parts that run as separate thread blocks and are merged afterwards.
+        pl->max_parts = 1;
+        if (!pairs.empty() && (int)pairs.size() * Hkv < kSplitTargetBlocks) {
+            int longest = 1;
+            for (auto &pr : pairs) longest = std::max(longest, steps_of(pr.second >= 0 ? pr.second : pr.first));
+            const int want = (kSplitTargetBlocks + (int)pairs.size() * Hkv - 1) / ((int)pairs.size() * Hkv);
+            pl->max_parts = std::max(1, std::min({want, kSplitMaxParts, longest / kSplitMinSteps}));
+        }
+        pl->combine.clear();
+        for (auto &pr : pairs) {
+            const int32_t a = pr.first, b2 = pr.second;
+            const int sa = steps_of(a), sl = steps_of(b2 >= 0 ? b2 : a);       // sa <= sl: positions ascend
+            const int parts = std::max(1, std::min(pl->max_parts, sl / kSplitMinSteps));
+            const int chunk = (sl + parts - 1) / parts;
+            for (int h = 0; h < Hkv; ++h) {
+                int parts_a = 0, parts_b = 0;
+                for (int p2 = 0; p2 < parts; ++p2) {
+                    const int sb = p2 * chunk, se = std::min(sl, sb + chunk);
+                    if (sb >= se) break;
+                    if (b2 < 0 || sb < sa) {
+                        pl->work.push_back({a, b2, h, sb, se, p2, parts, 0});
+                        ++parts_a;
+                        if (b2 >= 0) ++parts_b;
+                    } else {
+                        pl->work.push_back({b2, -1, h, sb, se, p2, parts, 0});   // tile a is already finished
+                        ++parts_b;
+                    }
+                }
+                if (parts > 1) {
+                    pl->combine.push_back({a, h, parts_a, 0});
+                    if (b2 >= 0) pl->combine.push_back({b2, h, parts_b, 0});
+                }
+            }
+        }
         auto cost = [&](const AttnWork &w) {
-            int c = (pl->tiles[w.tile_a].kv_len + page - 1) / page;
-            if (w.tile_b >= 0) c += (pl->tiles[w.tile_b].kv_len + page - 1) / page;
+            int c = std::min(w.step_end, steps_of(w.tile_a)) - w.step_begin;
+            if (w.tile_b >= 0) c += std::min(w.step_end, steps_of(w.tile_b)) - w.step_begin;
             return c;
         };
         auto sort_items = [&](std::vector<AttnWork>::iterator first_it, std::vector<AttnWork>::iterator last_it) {
@@ -295,6 +331,12 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
         for (int c = 0; c < used_chunks; ++c) pl->chunk_work_off[c + 1] += pl->chunk_work_off[c];
         for (int c = 0; c < used_chunks; ++c)
             sort_items(pl->work_chunked.begin() + pl->chunk_work_off[c], pl->work_chunked.begin() + pl->chunk_work_off[c + 1]);
+        std::stable_sort(pl->combine.begin(), pl->combine.end(), [&](const CombineItem &x, const CombineItem &y) {
+            return chunk_of[pl->tiles[x.tile].req] < chunk_of[pl->tiles[y.tile].req];
+        });
+        pl->chunk_combine_off.assign(used_chunks + 1, 0);
+        for (const CombineItem &ci : pl->combine) ++pl->chunk_combine_off[chunk_of[pl->tiles[ci.tile].req] + 1];
+        for (int c = 0; c < used_chunks; ++c) pl->chunk_combine_off[c + 1] += pl->chunk_combine_off[c];
         // Longest first in coarse cost bands; inside a band, items of one (request, KV head) stay
         // together, so thread blocks that run at the same time stream the same K/V pages and find
         // them in L2.

@@ -14,6 +14,9 @@ namespace tessera {
 constexpr int kGatherItemTokens = 32;   // token rows per thread block of the gather kernel
 constexpr int kAttnTileRows = 128;      // query rows (tokens x grouped heads) per tcgen05 tile
 constexpr bool kHaveTensorCoreKernel = true;
+constexpr int kSplitTargetBlocks = 148;  // split-KV aims at about this many thread blocks when a batch has fewer items
+constexpr int kSplitMinSteps = 4;        // never split below this many 128-key steps per part
+constexpr int kSplitMaxParts = 8;
 constexpr int kHostChunks = 4;          // request chunks of the host-buffer entry point's copy / compute pipeline
 constexpr int kAttnCostBands = 16;      // cost bands of the attention work list (longest band first)
 
@@ -31,8 +34,15 @@ struct AttnTile {
 
 // One thread block of the tcgen05 attention kernel: KV head `kvh` of query tiles tile_a and tile_b
 // (consecutive tiles of one request; tile_b = -1 when the request has an odd tile left over).
+// With split-KV the item covers only the 128-key steps [step_begin, step_end) and is part `part` of
+// `n_parts`; a part in which tile_a would have nothing to do names the longer tile alone.
 struct AttnWork {
-    int32_t tile_a, tile_b, kvh, n_steps;
+    int32_t tile_a, tile_b, kvh, step_begin, step_end, part, n_parts, pad;
+};
+
+// One (query tile, KV head) whose partial results have to be merged after a split-KV launch.
+struct CombineItem {
+    int32_t tile, kvh, n_parts, pad;
 };
 
 struct DeviceTables {
@@ -48,6 +58,9 @@ struct DeviceTables {
     AttnTile *tiles = nullptr;
     AttnWork *work = nullptr;      // tcgen05 work items, longest first
     AttnWork *work_chunked = nullptr;  // the same items grouped by request chunk (host-buffer entry)
+    CombineItem *combine = nullptr;    // (tile, head) pairs to merge, grouped by request chunk
+    float *ws_o = nullptr;             // split-KV partials: [slot][128 rows][128] unnormalised O ...
+    float2 *ws_ml = nullptr;           // ... and [slot][128] (reference maximum in log2 units, sum)
     int32_t *seq_len = nullptr;    // [batch]
     int32_t *status = nullptr;     // device status word(s)
     // staging for the host-buffer entry point (allocated on first use)
@@ -77,6 +90,9 @@ struct tessera_plan {
     // The host-buffer entry point pipelines copies against compute over chunks of whole requests.
     std::vector<tessera::AttnWork> work_chunked;   // items of chunk c: [chunk_work_off[c], chunk_work_off[c+1])
     std::vector<int32_t> chunk_work_off, chunk_row_off;   // [n_chunks + 1]; rows = recompute rows
+    std::vector<tessera::CombineItem> combine;     // grouped by chunk: [chunk_combine_off[c], chunk_combine_off[c+1])
+    std::vector<int32_t> chunk_combine_off;
+    int32_t max_parts = 1;                         // split-KV parts per item (1 = no split)
     int32_t attn_kernel = 0;
     int32_t tile_tokens = 0;
 
