@@ -170,7 +170,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     // Registers move from the producer / MMA warp group to the softmax warps, which hold a whole
     // 128-column row of S plus the packed probabilities.
     if (warp >= 8) {
-    reg_dealloc<56>();
+    reg_dealloc<80>();
     if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
@@ -294,7 +294,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         }
     }
     } else {
-        reg_alloc<224>();
+        reg_alloc<208>();
         // ------------------------------------------------------------------ softmax + epilogue
         // All eight warps work on ONE tile at a time and alternate between the tiles: warps 0-3 take
         // columns 0-63 of a row, warps 4-7 columns 64-127 (warp w and w + 4 share TMEM lanes).  The
@@ -431,9 +431,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int q = 0; q < n_tiles; ++q) {
             const AttnTile &t = q ? t1 : t0;
             const float l_tot = l_row[q] + l_xchg[(q * 2 + (h ^ 1)) * 128 + row];
-            if (wk.n_parts > 1) {
+            const AttnWork wke = work[blockIdx.x];     // re-read here rather than kept in registers through the loop
+            if (wke.n_parts > 1) {
                 // split-KV part: unnormalised accumulator, reference maximum and sum go to the workspace
-                const size_t slot = ((size_t)(q ? wk.tile_b : wk.tile_a) * H_kv + kvh) * max_parts + wk.part;
+                const size_t slot = ((size_t)(q ? wke.tile_b : wke.tile_a) * H_kv + kvh) * max_parts + wke.part;
                 float *po = ws_o + (slot * kRows + row) * kD + h * 64;
                 const uint32_t tOp = tmem + kTmemO + q * 128 + h * 64 + lane_base;
 #pragma unroll
