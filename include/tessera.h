@@ -221,6 +221,17 @@ TESSERA_API int32_t tessera_rope_shift_static(const tessera_model_cfg *cfg, void
                                               const int32_t *slot_shift, int32_t n_slots, const int32_t *shifts,
                                               int32_t n_shifts, void *stream);
 
+/*
+ * Diagnostic (the paper has no counterpart): exercises the bounded wait that every kernel of this
+ * library uses around its mbarriers.  Launches one small thread block that waits on a barrier nobody
+ * arrives on; the wait must give up after max_cycles SM cycles (1 .. 2e9), record code 42 and let the
+ * kernel end normally.  Synchronises `stream`.  Returns TESSERA_DEVICE_TIMEOUT when the wait ran out
+ * as intended (code_out = 42), TESSERA_OK if it did not (a defect).  cycles_out (host, nullable, 3
+ * entries): cycles spent in the first wait, cycles spent in a second wait issued after the abort flag
+ * was up (must be small), and a bit mask of waits that reported success (must be 0).
+ */
+TESSERA_API int32_t tessera_selftest_bounded_wait(int64_t max_cycles, int32_t *code_out, int64_t *cycles_out, void *stream);
+
 /* Copies the calling thread's last error text into buf (host); returns its length. */
 TESSERA_API int32_t tessera_last_error(char *buf, int32_t len);
 

@@ -54,7 +54,7 @@ class PlanInfo(ctypes.Structure):
 
 EXPORTS = ["tessera_plan_create", "tessera_plan_destroy", "tessera_plan_block_table", "tessera_plan_get_info",
            "tessera_plan_status", "tessera_kv_compose", "tessera_rope_shift", "tessera_partial_prefill_attn",
-           "tessera_composed_prefill_host", "tessera_rope_shift_static", "tessera_last_error",
+           "tessera_composed_prefill_host", "tessera_rope_shift_static", "tessera_selftest_bounded_wait", "tessera_last_error",
            "tessera_launch_count"]
 
 _vp = ctypes.c_void_p
@@ -70,6 +70,7 @@ _lib.tessera_partial_prefill_attn.argtypes = [_vp] * 9
 _lib.tessera_composed_prefill_host.argtypes = [_vp] * 9
 _lib.tessera_rope_shift_static.argtypes = [ctypes.POINTER(ModelCfg), _vp, _vp, _vp, ctypes.c_int32, _I32P,
                                            ctypes.c_int32, _vp]
+_lib.tessera_selftest_bounded_wait.argtypes = [ctypes.c_int64, _I32P, ctypes.POINTER(ctypes.c_int64), _vp]
 _lib.tessera_last_error.argtypes = [ctypes.c_char_p, ctypes.c_int32]
 _lib.tessera_launch_count.argtypes = []
 _lib.tessera_launch_count.restype = ctypes.c_int64
@@ -193,6 +194,14 @@ class Plan:
             self.destroy()
         except Exception:
             pass
+
+
+def selftest_bounded_wait(max_cycles: int, stream=None):
+    """tessera_selftest_bounded_wait: returns (status, code, [cycles first wait, cycles second wait, success mask])."""
+    code = ctypes.c_int32(0)
+    cyc = (ctypes.c_int64 * 3)()
+    st = _lib.tessera_selftest_bounded_wait(int(max_cycles), ctypes.byref(code), cyc, _stream(stream))
+    return int(st), int(code.value), [int(x) for x in cyc]
 
 
 STATIC_MAX_SHIFTS = 512

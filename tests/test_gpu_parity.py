@@ -226,3 +226,15 @@ def test_split_kv_single_request_with_wide_tiles():
     gu.check_attention(g, asm, use_pool_k=True)
     # same answer as the generic kernel's shape-independent definition: compare against config-2 style oracle only
     assert tb.Plan(w, host_only=True).info.n_attn_items > 8 * 2      # the items really were split
+
+
+def test_bounded_wait_gives_up_and_leaves_the_context_usable():
+    """A wait on a barrier that nobody completes must run out, report its code and return: the same
+    mechanism guards every mbarrier wait of the attention kernel."""
+    st, code, cyc = tb.selftest_bounded_wait(3_000_000)            # about 1.5 ms of SM cycles
+    assert st == tb.DEVICE_TIMEOUT and code == 42
+    assert 3_000_000 <= cyc[0] < 30_000_000                          # gave up after the limit, not much later
+    assert cyc[1] < 100_000 and cyc[2] == 0                          # later waits return at once, none "succeeded"
+    g = gu.run_layer(wl.config(1))                                   # the context is still fine
+    assert g.status == 0
+    gu.check_attention(g, gu.check_assembled(g)[0])
