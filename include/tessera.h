@@ -92,6 +92,11 @@ typedef struct tessera_compose_desc {
                                            its first source page; default 0.  Lets a unit be read out of the
                                            middle of another request's pages; it then spans
                                            ceil((offset + len) / page_size) source pages                 */
+    int32_t num_source_pages;           /* 0 (default): unit_pages index the destination pool.  > 0: the
+                                           cached units live in a SEPARATE source pool of this many pages
+                                           (same page layout) - the node's pinned host-memory unit cache of
+                                           Sec. 4 / 5.3 "local hit", or any other device-visible buffer;
+                                           such a plan is executed with tessera_kv_compose_from           */
     const int32_t *unit_target_stride;  /* [n_units] 1 (default): token i is rotated for position
                                            target_pos + i; 0: every token is rotated for position
                                            target_pos (with target_pos = 0: written without rotation)     */
@@ -160,6 +165,18 @@ TESSERA_API int32_t tessera_plan_status(tessera_plan *plan, int32_t *detail, voi
  * of a finished request (unit_src_offset) and whose unit_target_stride is 0 writes the un-rotated form.
  */
 TESSERA_API int32_t tessera_kv_compose(const tessera_plan *plan, void *k_pool, void *v_pool, uint32_t flags, void *stream);
+
+/*
+ * Local-hit path of Sec. 5.3: the cached units are copied out of a separate source pool - the
+ * node's PINNED HOST-MEMORY unit cache, read by the kernel straight over the interconnect (the memory
+ * must be device-addressable: cudaHostAlloc / cudaHostRegister), or another device buffer - into the
+ * request's destination pages in k_pool / v_pool, with the same flags and arithmetic as
+ * tessera_kv_compose.  The plan must have been created with desc.num_source_pages > 0, and such a plan
+ * is refused by tessera_kv_compose.  k_src, v_src: [num_source_pages][page_size][H_kv][D] bf16,
+ * 16-byte aligned, never written.  Throughput is bounded by the link to the source memory, not by HBM.
+ */
+TESSERA_API int32_t tessera_kv_compose_from(const tessera_plan *plan, const void *k_src, const void *v_src,
+                                            void *k_pool, void *v_pool, uint32_t flags, void *stream);
 
 /*
  * "Applying RoPE to the keys at their new positions" (Sec. 5.3; the fused placement kernel of

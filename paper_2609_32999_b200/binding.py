@@ -42,7 +42,7 @@ class ComposeDesc(ctypes.Structure):
                 ("unit_cached_pos", _I32P), ("unit_cached_stride", _I32P), ("unit_target_pos", _I32P),
                 ("unit_page_off", _I32P), ("unit_pages", _I32P), ("recompute_off", _I32P),
                 ("recompute_pos", _I32P), ("free_pages", _I32P), ("n_free", ctypes.c_int32),
-                ("unit_src_offset", _I32P), ("unit_target_stride", _I32P)]
+                ("unit_src_offset", _I32P), ("num_source_pages", ctypes.c_int32), ("unit_target_stride", _I32P)]
 
 
 class PlanInfo(ctypes.Structure):
@@ -53,7 +53,7 @@ class PlanInfo(ctypes.Structure):
 
 
 EXPORTS = ["tessera_plan_create", "tessera_plan_destroy", "tessera_plan_block_table", "tessera_plan_get_info",
-           "tessera_plan_status", "tessera_kv_compose", "tessera_rope_shift", "tessera_partial_prefill_attn",
+           "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_rope_shift", "tessera_partial_prefill_attn",
            "tessera_composed_prefill_host", "tessera_rope_shift_static", "tessera_selftest_bounded_wait", "tessera_last_error",
            "tessera_launch_count"]
 
@@ -65,6 +65,7 @@ _lib.tessera_plan_block_table.argtypes = [_vp, ctypes.POINTER(_I32P), ctypes.POI
 _lib.tessera_plan_get_info.argtypes = [_vp, ctypes.POINTER(PlanInfo)]
 _lib.tessera_plan_status.argtypes = [_vp, _I32P, _vp]
 _lib.tessera_kv_compose.argtypes = [_vp, _vp, _vp, ctypes.c_uint32, _vp]
+_lib.tessera_kv_compose_from.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_uint32, _vp]
 _lib.tessera_rope_shift.argtypes = [_vp, _vp, _vp]
 _lib.tessera_partial_prefill_attn.argtypes = [_vp] * 9
 _lib.tessera_composed_prefill_host.argtypes = [_vp] * 9
@@ -137,8 +138,9 @@ class Plan:
                        int(sh.rope_pairing), float(sh.sm_scale))
         opt = [None if getattr(w, f, None) is None else _arr(getattr(w, f))
                for f in ("unit_src_offset", "unit_target_stride")]
-        desc = ComposeDesc(len(a[0]), *[_ptr(x) for x in a[:11]], len(a[10]),
-                           *[None if x is None else _ptr(x) for x in opt])
+        op = [None if x is None else _ptr(x) for x in opt]
+        desc = ComposeDesc(len(a[0]), *[_ptr(x) for x in a[:11]], len(a[10]), op[0],
+                           int(getattr(w, "num_source_pages", 0) or 0), op[1])
         self._opt = opt
         self._h = _vp()
         self.host_only = host_only
@@ -170,6 +172,11 @@ class Plan:
     def kv_compose(self, k_pool, v_pool, fuse_rope: bool = True, stream=None) -> None:
         _check(_lib.tessera_kv_compose(self._h, _dev(k_pool), _dev(v_pool), FUSE_ROPE if fuse_rope else 0,
                                        _stream(stream)))
+
+    def kv_compose_from(self, k_src, v_src, k_pool, v_pool, fuse_rope: bool = True, stream=None) -> None:
+        """Sources in a separate pool (pinned host tensors or device tensors), destinations in the pools."""
+        _check(_lib.tessera_kv_compose_from(self._h, _dev(k_src), _dev(v_src), _dev(k_pool), _dev(v_pool),
+                                            FUSE_ROPE if fuse_rope else 0, _stream(stream)))
 
     def rope_shift(self, k_pool, stream=None) -> None:
         _check(_lib.tessera_rope_shift(self._h, _dev(k_pool), _stream(stream)))

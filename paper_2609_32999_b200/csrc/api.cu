@@ -250,7 +250,22 @@ int32_t tessera_kv_compose(const tessera_plan *pl, void *k_pool, void *v_pool, u
     if (flags & ~uint32_t(TESSERA_FUSE_ROPE)) return set_error(TESSERA_INVALID_ARG, "unknown compose flag");
     if (!k_pool || !v_pool || misaligned(k_pool) || misaligned(v_pool))
         return set_error(TESSERA_INVALID_ARG, "k_pool / v_pool must be non-null and 16-byte aligned");
-    TS_CUDA(launch_gather(pl, k_pool, v_pool, (flags & TESSERA_FUSE_ROPE) ? GatherMode::kCopyRotate : GatherMode::kCopy,
+    if (pl->num_source_pages > 0)
+        return set_error(TESSERA_INVALID_ARG, "this plan reads a separate source pool: use tessera_kv_compose_from");
+    TS_CUDA(launch_gather(pl, k_pool, v_pool, k_pool, v_pool, (flags & TESSERA_FUSE_ROPE) ? GatherMode::kCopyRotate : GatherMode::kCopy,
+                          static_cast<cudaStream_t>(stream)));
+    return TESSERA_OK;
+}
+
+int32_t tessera_kv_compose_from(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
+                                uint32_t flags, void *stream) {
+    if (int32_t rc = check_device_plan(pl)) return rc;
+    if (flags & ~uint32_t(TESSERA_FUSE_ROPE)) return set_error(TESSERA_INVALID_ARG, "unknown compose flag");
+    if (pl->num_source_pages <= 0)
+        return set_error(TESSERA_INVALID_ARG, "the plan was created without a separate source pool (desc.num_source_pages)");
+    if (!k_pool || !v_pool || !k_src || !v_src || misaligned(k_pool) || misaligned(v_pool) || misaligned(k_src) || misaligned(v_src))
+        return set_error(TESSERA_INVALID_ARG, "k_src / v_src / k_pool / v_pool must be non-null and 16-byte aligned");
+    TS_CUDA(launch_gather(pl, k_src, v_src, k_pool, v_pool, (flags & TESSERA_FUSE_ROPE) ? GatherMode::kCopyRotate : GatherMode::kCopy,
                           static_cast<cudaStream_t>(stream)));
     return TESSERA_OK;
 }
@@ -258,7 +273,7 @@ int32_t tessera_kv_compose(const tessera_plan *pl, void *k_pool, void *v_pool, u
 int32_t tessera_rope_shift(const tessera_plan *pl, void *k_pool, void *stream) {
     if (int32_t rc = check_device_plan(pl)) return rc;
     if (!k_pool || misaligned(k_pool)) return set_error(TESSERA_INVALID_ARG, "k_pool must be non-null and 16-byte aligned");
-    TS_CUDA(launch_gather(pl, k_pool, k_pool, GatherMode::kShiftInPlace, static_cast<cudaStream_t>(stream)));
+    TS_CUDA(launch_gather(pl, k_pool, k_pool, k_pool, k_pool, GatherMode::kShiftInPlace, static_cast<cudaStream_t>(stream)));
     return TESSERA_OK;
 }
 
@@ -279,6 +294,8 @@ int32_t tessera_composed_prefill_host(tessera_plan *pl, void *k_pool, void *v_po
     if (int32_t rc = check_device_plan(pl)) return rc;
     if (!k_pool || !v_pool || misaligned(k_pool) || misaligned(v_pool))
         return set_error(TESSERA_INVALID_ARG, "k_pool / v_pool must be non-null and 16-byte aligned");
+    if (pl->num_source_pages > 0)
+        return set_error(TESSERA_INVALID_ARG, "this plan reads a separate source pool: compose with tessera_kv_compose_from");
     if (pl->n_q > 0 && (!q_host || !k_new_host || !v_new_host || !out_host))
         return set_error(TESSERA_INVALID_ARG, "q / k_new / v_new / out host buffers must be non-null");
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -295,7 +312,7 @@ int32_t tessera_composed_prefill_host(tessera_plan *pl, void *k_pool, void *v_po
         TS_CUDA(cudaMemsetAsync(d.st_q, 0, q_bytes, st));   // rows of later chunks are read (and discarded) as tile padding
     }
     if (pl->n_q == 0) {
-        TS_CUDA(launch_gather(pl, k_pool, v_pool, GatherMode::kCopyRotate, st));
+        TS_CUDA(launch_gather(pl, k_pool, v_pool, k_pool, v_pool, GatherMode::kCopyRotate, st));
         TS_CUDA(cudaStreamSynchronize(st));
         return TESSERA_OK;
     }
@@ -321,7 +338,7 @@ int32_t tessera_composed_prefill_host(tessera_plan *pl, void *k_pool, void *v_po
         }
         TS_CUDA(cudaEventRecord(pl->ev_in[c], pl->s_in));
     }
-    TS_CUDA(launch_gather(pl, k_pool, v_pool, GatherMode::kCopyRotate, st));
+    TS_CUDA(launch_gather(pl, k_pool, v_pool, k_pool, v_pool, GatherMode::kCopyRotate, st));
     for (int c = 0; c < n_chunks; ++c) {
         const size_t r0 = pl->chunk_row_off[c], rows = pl->chunk_row_off[c + 1] - r0;
         TS_CUDA(cudaStreamWaitEvent(st, pl->ev_in[c], 0));

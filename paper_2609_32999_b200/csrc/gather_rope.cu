@@ -57,7 +57,7 @@ constexpr int kThreads = 256;
 // same two chunks of the V row.  IN_PLACE: source = destination, K only (the standalone shift).
 template <int D, bool DO_V, bool ROTATE, bool IN_PLACE>
 __global__ void __launch_bounds__(kThreads)
-gather_rope_kernel(uint4 *__restrict__ k_pool, uint4 *__restrict__ v_pool,
+gather_rope_kernel(const uint4 *k_src, const uint4 *v_src, uint4 *k_pool, uint4 *v_pool,
                    const int32_t *__restrict__ g_src, const int32_t *__restrict__ g_dst,
                    const GatherItem *__restrict__ items, const float2 *__restrict__ rope, int H_kv) {
     constexpr int CPH = D / 16;          // pair-chunks per head
@@ -107,12 +107,12 @@ gather_rope_kernel(uint4 *__restrict__ k_pool, uint4 *__restrict__ v_pool,
                 klo[u] = ldg_plain(k_pool + so);
                 khi[u] = ldg_plain(k_pool + so + HALF);
             } else {
-                klo[u] = ldg_stream(k_pool + so);
-                khi[u] = ldg_stream(k_pool + so + HALF);
+                klo[u] = ldg_stream(k_src + so);
+                khi[u] = ldg_stream(k_src + so + HALF);
             }
             if (DO_V) {
-                vlo[u] = ldg_stream(v_pool + so);
-                vhi[u] = ldg_stream(v_pool + so + HALF);
+                vlo[u] = ldg_stream(v_src + so);
+                vhi[u] = ldg_stream(v_src + so + HALF);
             }
         }
 #pragma unroll
@@ -157,22 +157,25 @@ scatter_fresh_kernel(uint4 *__restrict__ k_pool, uint4 *__restrict__ v_pool,
 }
 
 template <int D>
-cudaError_t launch_gather_d(const tessera_plan *pl, void *k_pool, void *v_pool, GatherMode mode, cudaStream_t st) {
+cudaError_t launch_gather_d(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
+                            GatherMode mode, cudaStream_t st) {
     const int n = (int)pl->items.size();
     if (n == 0) return cudaSuccess;
     auto *kp = static_cast<uint4 *>(k_pool);
     auto *vp = static_cast<uint4 *>(v_pool);
+    auto *ks = static_cast<const uint4 *>(k_src);
+    auto *vs = static_cast<const uint4 *>(v_src);
     const DeviceTables &d = pl->dev;
     const int H = pl->cfg.num_kv_heads;
     switch (mode) {
         case GatherMode::kCopy:
-            gather_rope_kernel<D, true, false, false><<<n, kThreads, 0, st>>>(kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            gather_rope_kernel<D, true, false, false><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
             break;
         case GatherMode::kCopyRotate:
-            gather_rope_kernel<D, true, true, false><<<n, kThreads, 0, st>>>(kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            gather_rope_kernel<D, true, true, false><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
             break;
         case GatherMode::kShiftInPlace:
-            gather_rope_kernel<D, false, true, true><<<n, kThreads, 0, st>>>(kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            gather_rope_kernel<D, false, true, true><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
             break;
     }
     count_launch();
@@ -181,9 +184,10 @@ cudaError_t launch_gather_d(const tessera_plan *pl, void *k_pool, void *v_pool, 
 
 }  // namespace
 
-cudaError_t launch_gather(const tessera_plan *pl, void *k_pool, void *v_pool, GatherMode mode, cudaStream_t st) {
-    return pl->cfg.head_dim == 128 ? launch_gather_d<128>(pl, k_pool, v_pool, mode, st)
-                                   : launch_gather_d<64>(pl, k_pool, v_pool, mode, st);
+cudaError_t launch_gather(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
+                          GatherMode mode, cudaStream_t st) {
+    return pl->cfg.head_dim == 128 ? launch_gather_d<128>(pl, k_src, v_src, k_pool, v_pool, mode, st)
+                                   : launch_gather_d<64>(pl, k_src, v_src, k_pool, v_pool, mode, st);
 }
 
 cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_pool, const void *k_new,

@@ -54,6 +54,9 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
     pl->cfg.inv_freq = nullptr;
     pl->sm_scale = cfg->sm_scale != 0.f ? cfg->sm_scale : (float)(1.0 / std::sqrt((double)D));
     pl->num_pool_pages = num_pool_pages;
+    if (d->num_source_pages < 0) return fail(TESSERA_INVALID_ARG, "negative num_source_pages");
+    if ((int64_t)d->num_source_pages * B > (int64_t)INT32_MAX) return fail(TESSERA_UNSUPPORTED_SHAPE, "source pool has more than 2^31 slots");
+    pl->num_source_pages = d->num_source_pages;
     pl->batch = d->batch;
 
     const int batch = d->batch;
@@ -111,8 +114,9 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
     const int n_src_pages = n_units ? d->unit_page_off[n_units] : 0;
     for (int k = 0; k < n_src_pages; ++k) {
         int pg = d->unit_pages[k];
-        if (pg < 0 || pg >= num_pool_pages) return fail(TESSERA_PAGE_OUT_OF_RANGE, fmt("source page %ld outside pool of %ld pages", pg, num_pool_pages));
-        page_use[pg] = 1;
+        const int src_limit = d->num_source_pages > 0 ? d->num_source_pages : num_pool_pages;
+        if (pg < 0 || pg >= src_limit) return fail(TESSERA_PAGE_OUT_OF_RANGE, fmt("source page %ld outside pool of %ld pages", pg, src_limit));
+        if (d->num_source_pages == 0) page_use[pg] = 1;    // a separate source pool cannot alias destinations
     }
     for (int64_t k = 0; k < need_pages; ++k) {
         int pg = pl->pages[k];

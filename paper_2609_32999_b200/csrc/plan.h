@@ -75,6 +75,7 @@ struct tessera_plan {
     std::vector<double> inv_freq;          // [D/2], always filled
     float sm_scale = 0.f;
     int32_t num_pool_pages = 0;
+    int32_t num_source_pages = 0;          // > 0: cached units are read from a separate source pool
     int32_t batch = 0;
     bool host_only = false;
     int device = -1;

@@ -54,6 +54,7 @@ class Workload:
     n_layers: int = 1
     unit_src_offset: Optional[np.ndarray] = None     # [n_units] token 0's offset inside its first source page
     unit_target_stride: Optional[np.ndarray] = None  # [n_units] 0 = every token rotated for target_pos
+    num_source_pages: int = 0                        # > 0: unit_pages index a separate source pool (host tier)
 
     @property
     def batch(self) -> int:

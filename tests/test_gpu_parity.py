@@ -238,3 +238,43 @@ def test_bounded_wait_gives_up_and_leaves_the_context_usable():
     g = gu.run_layer(wl.config(1))                                   # the context is still fine
     assert g.status == 0
     gu.check_attention(g, gu.check_assembled(g)[0])
+
+
+def test_host_tier_compose_reads_a_pinned_host_pool():
+    """Local-hit path: the cached units sit in pinned host memory (a separate source pool) and the
+    gather kernel reads them over the interconnect; the device copies of the sources are wiped first."""
+    import copy
+    w = wl.config(3, requests_override=4)
+    dev = "cuda:0"
+    t = wl.make_tensors(w, device=dev, seed=12)
+    host_k, host_v = t.k_pool.cpu().pin_memory(), t.v_pool.cpu().pin_memory()
+    w2 = copy.copy(w)
+    w2.num_source_pages = w.num_pool_pages
+    plan = tb.Plan(w2)
+    pv = torch.tensor(gu.POISON, dtype=torch.int16, device=dev).view(torch.bfloat16)
+    t.k_pool[:] = pv
+    t.v_pool[:] = pv
+    with pytest.raises(tb.TesseraError):
+        plan.kv_compose(t.k_pool, t.v_pool)                  # such a plan needs the _from entry point
+    plan.kv_compose_from(host_k, host_v, t.k_pool, t.v_pool)
+    torch.cuda.synchronize()
+    g = gu.GpuRun()
+    g.w, g.t, g.plan = w, t, plan
+    g.page_off, g.pages, g.src_slot = plan.block_table()
+    g.k_before, g.v_before = orc.bits(host_k), orc.bits(host_v)
+    g.k_after, g.v_after = orc.bits(t.k_pool), orc.bits(t.v_pool)
+    g.kn_bits, g.vn_bits = orc.bits(t.k_new), orc.bits(t.v_new)
+    gu.check_placement(g)
+    asm, kmx, kmean = gu.check_assembled(g, scattered=False)
+    # nothing but destination pages was written
+    mask = np.ones(w.num_pool_pages, bool)
+    mask[g.pages] = False
+    assert np.all(g.k_after[mask] == gu.POISON) and np.all(g.v_after[mask] == gu.POISON)
+    # and the attention path works on top of it
+    out = torch.empty_like(t.q)
+    plan.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, out, None)
+    torch.cuda.synchronize()
+    g.k_after, g.v_after = orc.bits(t.k_pool), orc.bits(t.v_pool)
+    g.q_bits, g.out_f, g.lse_f = orc.bits(t.q), out.float().cpu().numpy().astype(np.float64), None
+    asm, _, _ = gu.check_assembled(g)
+    gu.check_attention(g, asm)
