@@ -278,3 +278,33 @@ def test_host_tier_compose_reads_a_pinned_host_pool():
     g.q_bits, g.out_f, g.lse_f = orc.bits(t.q), out.float().cpu().numpy().astype(np.float64), None
     asm, _, _ = gu.check_assembled(g)
     gu.check_attention(g, asm)
+
+
+@pytest.mark.parametrize("hq,hkv", [(16, 8), (16, 1), (2, 2)])
+def test_other_group_sizes_on_the_tensor_core_path(hq, hkv):
+    """g = 2, 16 and 1 query heads per KV head (tiles of 64, 8 and 128 tokens)."""
+    w = wl.adversarial(seed=20 + hq, shape=wl.ModelShape(hq, hkv, 128, 64, 500000.0))
+    g, _ = _full_check(w)
+    assert g.plan.info.attn_kernel == 1
+
+
+def test_batches_without_queries_or_without_requests():
+    shape = wl.ModelShape(32, 8, 128, 64, 500000.0)
+    dev = "cuda:0"
+    # every position cached, nothing recomputed: attention is a no-op that still returns OK
+    w = wl.build_workload("noq", shape, [[wl.unit(100, "a"), wl.unit(70, "b", cached_pos=5)]], np.random.default_rng(1))
+    g = gu.run_layer(w)
+    assert g.status == 0 and w.n_q == 0
+    gu.check_assembled(g)
+    gu.check_untouched(g)
+    # empty batch
+    w = wl.build_workload("empty", shape, [], np.random.default_rng(1))
+    t = wl.make_tensors(w, device=dev)
+    plan = tb.Plan(w)
+    before = t.k_pool.clone()
+    plan.kv_compose(t.k_pool, t.v_pool)
+    plan.rope_shift(t.k_pool)
+    plan.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, torch.empty_like(t.q), None)
+    plan.composed_prefill_host(t.k_pool, t.v_pool, t.q.cpu(), t.k_new.cpu(), t.v_new.cpu(), t.q.cpu(), None)
+    torch.cuda.synchronize()
+    assert torch.equal(before, t.k_pool) and plan.status() == 0
