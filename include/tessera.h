@@ -187,6 +187,16 @@ TESSERA_API int32_t tessera_kv_compose_from(const tessera_plan *plan, const void
 TESSERA_API int32_t tessera_rope_shift(const tessera_plan *plan, void *k_pool, void *stream);
 
 /*
+ * Neighbour of the extend pass (Sec. 5.3 "Completing prefill"; Sec. 2.2: queries and keys are rotated,
+ * values are not): rotates, in place, the fresh queries q [n_q][H_q][D] and fresh keys k_new
+ * [n_q][H_kv][D] (device, bf16) of the recompute rows for their target positions recompute_pos[j].
+ * Either pointer may be NULL.  Angles, cosines and sines are evaluated in fp64 on the device and used
+ * as fp32; fp32 math, one round-to-nearest-even to bf16.  Call it when the caller hands over
+ * un-rotated projections; tessera_partial_prefill_attn itself expects rotated q and k_new.
+ */
+TESSERA_API int32_t tessera_rope_fresh(const tessera_plan *plan, void *q, void *k_new, void *stream);
+
+/*
  * Completing prefill (Sec. 5.3): the extend pass restricted to the recompute rows.
  *   1. writes k_new / v_new (device, [n_q][H_kv][D], keys already rotated at their target
  *      positions) into the rows' destination slots, overriding cached values - recomputed states

@@ -53,7 +53,7 @@ class PlanInfo(ctypes.Structure):
 
 
 EXPORTS = ["tessera_plan_create", "tessera_plan_destroy", "tessera_plan_block_table", "tessera_plan_get_info",
-           "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_rope_shift", "tessera_partial_prefill_attn",
+           "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_rope_shift", "tessera_rope_fresh", "tessera_partial_prefill_attn",
            "tessera_composed_prefill_host", "tessera_rope_shift_static", "tessera_selftest_bounded_wait", "tessera_last_error",
            "tessera_launch_count"]
 
@@ -67,6 +67,7 @@ _lib.tessera_plan_status.argtypes = [_vp, _I32P, _vp]
 _lib.tessera_kv_compose.argtypes = [_vp, _vp, _vp, ctypes.c_uint32, _vp]
 _lib.tessera_kv_compose_from.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_uint32, _vp]
 _lib.tessera_rope_shift.argtypes = [_vp, _vp, _vp]
+_lib.tessera_rope_fresh.argtypes = [_vp, _vp, _vp, _vp]
 _lib.tessera_partial_prefill_attn.argtypes = [_vp] * 9
 _lib.tessera_composed_prefill_host.argtypes = [_vp] * 9
 _lib.tessera_rope_shift_static.argtypes = [ctypes.POINTER(ModelCfg), _vp, _vp, _vp, ctypes.c_int32, _I32P,
@@ -180,6 +181,10 @@ class Plan:
 
     def rope_shift(self, k_pool, stream=None) -> None:
         _check(_lib.tessera_rope_shift(self._h, _dev(k_pool), _stream(stream)))
+
+    def rope_fresh(self, q, k_new, stream=None) -> None:
+        """Rotate fresh q / k_new rows in place for their target positions (either may be None)."""
+        _check(_lib.tessera_rope_fresh(self._h, _dev(q), _dev(k_new), _stream(stream)))
 
     def partial_prefill_attn(self, k_pool, v_pool, q, k_new, v_new, out, lse=None, stream=None) -> None:
         _check(_lib.tessera_partial_prefill_attn(self._h, _dev(k_pool), _dev(v_pool), _dev(q), _dev(k_new),

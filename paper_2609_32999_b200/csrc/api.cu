@@ -59,6 +59,7 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     const size_t o_comb = place<CombineItem>(off, pl->combine.size());
     const size_t o_seq = place<int32_t>(off, pl->seq_len.size());
     const size_t o_status = place<int32_t>(off, 4);
+    const size_t o_invf = place<double>(off, pl->inv_freq.size());
     // split-KV workspace: one slot per (tile, KV head, part)
     const size_t n_slots = pl->max_parts > 1 ? pl->tiles.size() * pl->cfg.num_kv_heads * pl->max_parts : 0;
     const size_t o_wsml = place<float2>(off, n_slots * kAttnTileRows);
@@ -80,6 +81,7 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     put(o_work, pl->work.data(), pl->work.size() * sizeof(AttnWork));
     put(o_workc, pl->work_chunked.data(), pl->work_chunked.size() * sizeof(AttnWork));
     put(o_comb, pl->combine.data(), pl->combine.size() * sizeof(CombineItem));
+    put(o_invf, pl->inv_freq.data(), pl->inv_freq.size() * sizeof(double));
     put(o_seq, pl->seq_len.data(), pl->seq_len.size() * 4);
     TS_CUDA(cudaMalloc(&d.blob, off));
     TS_CUDA(cudaMemcpyAsync(d.blob, hb, table_bytes, cudaMemcpyHostToDevice, st));
@@ -101,6 +103,7 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     d.ws_o = reinterpret_cast<float *>(db + o_wso);
     d.seq_len = reinterpret_cast<int32_t *>(db + o_seq);
     d.status = reinterpret_cast<int32_t *>(db + o_status);
+    d.inv_freq = reinterpret_cast<double *>(db + o_invf);
     return TESSERA_OK;
 }
 
@@ -274,6 +277,13 @@ int32_t tessera_rope_shift(const tessera_plan *pl, void *k_pool, void *stream) {
     if (int32_t rc = check_device_plan(pl)) return rc;
     if (!k_pool || misaligned(k_pool)) return set_error(TESSERA_INVALID_ARG, "k_pool must be non-null and 16-byte aligned");
     TS_CUDA(launch_gather(pl, k_pool, k_pool, k_pool, k_pool, GatherMode::kShiftInPlace, static_cast<cudaStream_t>(stream)));
+    return TESSERA_OK;
+}
+
+int32_t tessera_rope_fresh(const tessera_plan *pl, void *q, void *k_new, void *stream) {
+    if (int32_t rc = check_device_plan(pl)) return rc;
+    if (misaligned(q) || misaligned(k_new)) return set_error(TESSERA_INVALID_ARG, "q / k_new must be 16-byte aligned");
+    TS_CUDA(launch_rope_fresh(pl, q, k_new, static_cast<cudaStream_t>(stream)));
     return TESSERA_OK;
 }
 

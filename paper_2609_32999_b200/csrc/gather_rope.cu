@@ -156,6 +156,41 @@ scatter_fresh_kernel(uint4 *__restrict__ k_pool, uint4 *__restrict__ v_pool,
     }
 }
 
+// Rotates the fresh q and k_new rows of recompute row j for position q_pos[j] (Sec. 2.2 / 5.3).  One
+// thread block per row: the first D/2 threads evaluate cos / sin of (position x frequency) in fp64,
+// then every thread rotates pair-chunks exactly as the gather kernel does.
+template <int D>
+__global__ void __launch_bounds__(128)
+rope_fresh_kernel(uint4 *__restrict__ q, uint4 *__restrict__ k_new, const int32_t *__restrict__ q_pos,
+                  const double *__restrict__ inv_freq, int H_q, int H_kv) {
+    constexpr int CPH = D / 16, HALF = D / 16;
+    __shared__ float2 s_cs[D / 2];
+    const int j = blockIdx.x, tid = threadIdx.x;
+    if (tid < D / 2) {
+        double sn, cs;
+        sincos((double)q_pos[j] * inv_freq[tid], &sn, &cs);
+        s_cs[tid] = make_float2((float)cs, (float)sn);
+    }
+    __syncthreads();
+    const int c = tid % CPH;
+    float2 cr[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) cr[i] = s_cs[c * 8 + i];
+    for (int pass = 0; pass < 2; ++pass) {
+        uint4 *base = pass ? k_new : q;
+        const int heads = pass ? H_kv : H_q;
+        if (!base) continue;
+        uint4 *row = base + (size_t)j * heads * (D / 8);
+        for (int t = tid; t < heads * CPH; t += 128) {
+            uint4 *plo = row + (t / CPH) * (D / 8) + c, *phi = plo + HALF;
+            uint4 lo = *plo, hi = *phi;
+            rotate8(lo, hi, cr);
+            *plo = lo;
+            *phi = hi;
+        }
+    }
+}
+
 template <int D>
 cudaError_t launch_gather_d(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
                             GatherMode mode, cudaStream_t st) {
@@ -188,6 +223,19 @@ cudaError_t launch_gather(const tessera_plan *pl, const void *k_src, const void 
                           GatherMode mode, cudaStream_t st) {
     return pl->cfg.head_dim == 128 ? launch_gather_d<128>(pl, k_src, v_src, k_pool, v_pool, mode, st)
                                    : launch_gather_d<64>(pl, k_src, v_src, k_pool, v_pool, mode, st);
+}
+
+cudaError_t launch_rope_fresh(const tessera_plan *pl, void *q, void *k_new, cudaStream_t st) {
+    if (pl->n_q == 0 || (!q && !k_new)) return cudaSuccess;
+    const DeviceTables &d = pl->dev;
+    if (pl->cfg.head_dim == 128)
+        rope_fresh_kernel<128><<<(unsigned)pl->n_q, 128, 0, st>>>(static_cast<uint4 *>(q), static_cast<uint4 *>(k_new), d.q_pos,
+                                                                 d.inv_freq, pl->cfg.num_q_heads, pl->cfg.num_kv_heads);
+    else
+        rope_fresh_kernel<64><<<(unsigned)pl->n_q, 128, 0, st>>>(static_cast<uint4 *>(q), static_cast<uint4 *>(k_new), d.q_pos,
+                                                                d.inv_freq, pl->cfg.num_q_heads, pl->cfg.num_kv_heads);
+    count_launch();
+    return cudaGetLastError();
 }
 
 cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_pool, const void *k_new,

@@ -14,6 +14,8 @@ void count_launch();   // bumps the process-wide kernel-launch counter
 // separate source pool - and written to the plan's destination slots in (k_pool, v_pool).
 cudaError_t launch_gather(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
                           GatherMode mode, cudaStream_t st);
+// In-place rotation of the fresh q / k_new rows for their target positions (either may be null).
+cudaError_t launch_rope_fresh(const tessera_plan *pl, void *q, void *k_new, cudaStream_t st);
 // chunk < 0: the whole batch; otherwise only request chunk `chunk` (see tessera_plan::chunk_row_off).
 // k_new / v_new / q / out / lse always point at row 0 of the whole batch.
 cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_pool, const void *k_new,

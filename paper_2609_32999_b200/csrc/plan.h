@@ -63,6 +63,7 @@ struct DeviceTables {
     float2 *ws_ml = nullptr;           // ... and [slot][128] (reference maximum in log2 units, sum)
     int32_t *seq_len = nullptr;    // [batch]
     int32_t *status = nullptr;     // device status word(s)
+    double *inv_freq = nullptr;    // [D/2] rotary frequencies
     // staging for the host-buffer entry point (allocated on first use)
     void *st_q = nullptr, *st_k = nullptr, *st_v = nullptr, *st_o = nullptr;
     float *st_lse = nullptr;

@@ -13,7 +13,7 @@ MAX_ABS, MEAN_ABS = 2e-2, 2e-3          # tolerance of bf16 attention outputs an
 POISON = 0x7FC1                         # a NaN pattern no kernel produces
 
 
-class GpuRun:
+class LayerRun:
     pass
 
 
@@ -32,7 +32,7 @@ def run_layer(w, t=None, fuse=True, layer=0, seed=None, poison=True, with_lse=Tr
         pv = torch.tensor(POISON, dtype=torch.int16, device=dev).view(torch.bfloat16)
         t.k_pool[idx] = pv
         t.v_pool[idx] = pv
-    g = GpuRun()
+    g = LayerRun()
     g.w, g.t, g.plan = w, t, plan
     g.page_off, g.pages, g.src_slot = page_off, pages, src_slot
     g.k_before, g.v_before = orc.bits(t.k_pool).copy(), orc.bits(t.v_pool).copy()

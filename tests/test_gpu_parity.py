@@ -258,7 +258,7 @@ def test_host_tier_compose_reads_a_pinned_host_pool():
         plan.kv_compose(t.k_pool, t.v_pool)                  # such a plan needs the _from entry point
     plan.kv_compose_from(host_k, host_v, t.k_pool, t.v_pool)
     torch.cuda.synchronize()
-    g = gu.GpuRun()
+    g = gu.LayerRun()
     g.w, g.t, g.plan = w, t, plan
     g.page_off, g.pages, g.src_slot = plan.block_table()
     g.k_before, g.v_before = orc.bits(host_k), orc.bits(host_v)
@@ -308,3 +308,32 @@ def test_batches_without_queries_or_without_requests():
     plan.composed_prefill_host(t.k_pool, t.v_pool, t.q.cpu(), t.k_new.cpu(), t.v_new.cpu(), t.q.cpu(), None)
     torch.cuda.synchronize()
     assert torch.equal(before, t.k_pool) and plan.status() == 0
+
+
+@pytest.mark.parametrize("make", [lambda: wl.config(1), lambda: wl.config(3, requests_override=2),
+                                  lambda: wl.adversarial(seed=9, shape=wl.ModelShape(32, 8, 128, 64, 500000.0))])
+def test_rope_fresh_rotates_queries_and_keys_at_target_positions(make):
+    w = make()
+    dev = "cuda:0"
+    t = wl.make_tensors(w, device=dev, seed=44)
+    q0, k0 = orc.bf16_bits_to_f64(orc.bits(t.q)), orc.bf16_bits_to_f64(orc.bits(t.k_new))
+    plan = tb.Plan(w)
+    plan.rope_fresh(t.q, t.k_new)
+    plan.rope_fresh(None, None)                                     # nothing to do is fine
+    torch.cuda.synchronize()
+    q1, k1 = orc.bf16_bits_to_f64(orc.bits(t.q)), orc.bf16_bits_to_f64(orc.bits(t.k_new))
+    theta = w.shape.rope_theta
+    rng = np.random.default_rng(0)
+    errs = []
+    for j in rng.choice(w.n_q, size=min(w.n_q, 40), replace=False):
+        p = int(w.recompute_pos[j])
+        for h in range(w.shape.num_q_heads):
+            errs.append(np.abs(orc.rope_rotate(q0[j, h], p, theta) - q1[j, h]))
+        for h in range(w.shape.num_kv_heads):
+            errs.append(np.abs(orc.rope_rotate(k0[j, h], p, theta) - k1[j, h]))
+    e = np.concatenate(errs)
+    assert e.max() <= gu.MAX_ABS and e.mean() <= gu.MEAN_ABS
+    # position 0 rows are bit copies
+    zero = np.nonzero(w.recompute_pos == 0)[0]
+    for j in zero:
+        assert np.array_equal(q0[j], q1[j]) and np.array_equal(k0[j], k1[j])
