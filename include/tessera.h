@@ -61,7 +61,7 @@ typedef struct tessera_model_cfg {
     int32_t page_size;          /* tokens per storage block, a multiple of 8, at most 128      */
     double  rope_theta;         /* pair m turns by theta^(-2m/D) per position                  */
     const double *inv_freq;     /* host, optional [D/2]: overrides rope_theta when non-null     */
-    int32_t rope_pairing;       /* 0 = pair (m, m + D/2); other values: TESSERA_UNSUPPORTED_SHAPE */
+    int32_t rope_pairing;       /* 0 = pair (m, m + D/2) (Llama / Qwen); 1 = pair (2m, 2m + 1) (interleaved) */
     float   sm_scale;           /* softmax scale; 0 means 1/sqrt(D)                             */
 } tessera_model_cfg;
 

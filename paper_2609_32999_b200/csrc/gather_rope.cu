@@ -50,12 +50,42 @@ __device__ __forceinline__ void rotate8(uint4 &lo, uint4 &hi, const float2 *cs) 
     }
 }
 
+// Interleaved pairing: pair m = (element 2m, element 2m + 1).  One 16-byte chunk holds 4 whole pairs;
+// cs[0..3] are the (cos, sin) of the chunk's pairs.
+__device__ __forceinline__ void rotate4_interleaved(uint4 &v, const float2 *cs) {
+    uint32_t *w = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float x = __uint_as_float(w[i] << 16), y = __uint_as_float(w[i] & 0xffff0000u);
+        const float2 c = cs[i];
+        __nv_bfloat162 p = __floats2bfloat162_rn(fmaf(-y, c.y, x * c.x), fmaf(x, c.y, y * c.x));
+        w[i] = *reinterpret_cast<uint32_t *>(&p);
+    }
+}
+// Rotates the two chunks a task holds.  Half-split pairing: lo / hi are the two halves of 8 pairs and
+// cs = the 8 (cos, sin) of pairs 8c .. 8c+7.  Interleaved: lo holds pairs 4c .. 4c+3 (cs[0..3]) and hi,
+// D/2 elements later, pairs 4c + D/4 .. (cs[4..7]).
+template <bool INTERLEAVED>
+__device__ __forceinline__ void rotate_task(uint4 &lo, uint4 &hi, const float2 *cs) {
+    if (INTERLEAVED) {
+        rotate4_interleaved(lo, cs);
+        rotate4_interleaved(hi, cs + 4);
+    } else {
+        rotate8(lo, hi, cs);
+    }
+}
+// Index (within a D/2-entry cos/sin row) of entry i of the 8 a task with chunk index c needs.
+template <int D, bool INTERLEAVED>
+__device__ __forceinline__ int cs_index(int c, int i) {
+    return INTERLEAVED ? (i < 4 ? 4 * c + i : 4 * c + D / 4 + (i - 4)) : c * 8 + i;
+}
+
 constexpr int kThreads = 256;
 
 // One thread block per GatherItem.  A "task" is one rotary pair-chunk of one token row: the 16-byte
 // chunk holding elements [8c, 8c+8) of a head and its partner chunk D/2 elements later (K), plus the
 // same two chunks of the V row.  IN_PLACE: source = destination, K only (the standalone shift).
-template <int D, bool DO_V, bool ROTATE, bool IN_PLACE>
+template <int D, bool DO_V, bool ROTATE, bool IN_PLACE, bool INTERLEAVED>
 __global__ void __launch_bounds__(kThreads)
 gather_rope_kernel(const uint4 *k_src, const uint4 *v_src, uint4 *k_pool, uint4 *v_pool,
                    const int32_t *__restrict__ g_src, const int32_t *__restrict__ g_dst,
@@ -84,7 +114,7 @@ gather_rope_kernel(const uint4 *k_src, const uint4 *v_src, uint4 *k_pool, uint4 
     float2 cs[8];
     if (ROTATE && it.row_step == 0) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) cs[i] = s_rope[c * 8 + i];
+        for (int i = 0; i < 8; ++i) cs[i] = s_rope[cs_index<D, INTERLEAVED>(c, i)];
     }
 
     constexpr int U = 2;                 // tasks in flight per thread
@@ -125,13 +155,13 @@ gather_rope_kernel(const uint4 *k_src, const uint4 *v_src, uint4 *k_pool, uint4 
             if (ROTATE) {
                 if (it.row_step != 0) {
                     const int sr = it.row_step < 0 ? it.count - 1 - tok[u] : tok[u];
-                    const float2 *row = s_rope + (size_t)sr * (D / 2) + c * 8;
+                    const float2 *row = s_rope + (size_t)sr * (D / 2);
                     float2 cr[8];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) cr[i] = row[i];
-                    rotate8(klo[u], khi[u], cr);
+                    for (int i = 0; i < 8; ++i) cr[i] = row[cs_index<D, INTERLEAVED>(c, i)];
+                    rotate_task<INTERLEAVED>(klo[u], khi[u], cr);
                 } else {
-                    rotate8(klo[u], khi[u], cs);
+                    rotate_task<INTERLEAVED>(klo[u], khi[u], cs);
                 }
             }
             stg(k_pool + dsto[u], klo[u]);
@@ -159,7 +189,7 @@ scatter_fresh_kernel(uint4 *__restrict__ k_pool, uint4 *__restrict__ v_pool,
 // Rotates the fresh q and k_new rows of recompute row j for position q_pos[j] (Sec. 2.2 / 5.3).  One
 // thread block per row: the first D/2 threads evaluate cos / sin of (position x frequency) in fp64,
 // then every thread rotates pair-chunks exactly as the gather kernel does.
-template <int D>
+template <int D, bool INTERLEAVED>
 __global__ void __launch_bounds__(128)
 rope_fresh_kernel(uint4 *__restrict__ q, uint4 *__restrict__ k_new, const int32_t *__restrict__ q_pos,
                   const double *__restrict__ inv_freq, int H_q, int H_kv) {
@@ -175,7 +205,7 @@ rope_fresh_kernel(uint4 *__restrict__ q, uint4 *__restrict__ k_new, const int32_
     const int c = tid % CPH;
     float2 cr[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) cr[i] = s_cs[c * 8 + i];
+    for (int i = 0; i < 8; ++i) cr[i] = s_cs[cs_index<D, INTERLEAVED>(c, i)];
     for (int pass = 0; pass < 2; ++pass) {
         uint4 *base = pass ? k_new : q;
         const int heads = pass ? H_kv : H_q;
@@ -184,14 +214,14 @@ rope_fresh_kernel(uint4 *__restrict__ q, uint4 *__restrict__ k_new, const int32_
         for (int t = tid; t < heads * CPH; t += 128) {
             uint4 *plo = row + (t / CPH) * (D / 8) + c, *phi = plo + HALF;
             uint4 lo = *plo, hi = *phi;
-            rotate8(lo, hi, cr);
+            rotate_task<INTERLEAVED>(lo, hi, cr);
             *plo = lo;
             *phi = hi;
         }
     }
 }
 
-template <int D>
+template <int D, bool IL>
 cudaError_t launch_gather_d(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
                             GatherMode mode, cudaStream_t st) {
     const int n = (int)pl->items.size();
@@ -204,13 +234,13 @@ cudaError_t launch_gather_d(const tessera_plan *pl, const void *k_src, const voi
     const int H = pl->cfg.num_kv_heads;
     switch (mode) {
         case GatherMode::kCopy:
-            gather_rope_kernel<D, true, false, false><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            gather_rope_kernel<D, true, false, false, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
             break;
         case GatherMode::kCopyRotate:
-            gather_rope_kernel<D, true, true, false><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            gather_rope_kernel<D, true, true, false, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
             break;
         case GatherMode::kShiftInPlace:
-            gather_rope_kernel<D, false, true, true><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            gather_rope_kernel<D, false, true, true, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
             break;
     }
     count_launch();
@@ -221,19 +251,29 @@ cudaError_t launch_gather_d(const tessera_plan *pl, const void *k_src, const voi
 
 cudaError_t launch_gather(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
                           GatherMode mode, cudaStream_t st) {
-    return pl->cfg.head_dim == 128 ? launch_gather_d<128>(pl, k_src, v_src, k_pool, v_pool, mode, st)
-                                   : launch_gather_d<64>(pl, k_src, v_src, k_pool, v_pool, mode, st);
+    const bool il = pl->cfg.rope_pairing == 1;
+    if (pl->cfg.head_dim == 128)
+        return il ? launch_gather_d<128, true>(pl, k_src, v_src, k_pool, v_pool, mode, st)
+                  : launch_gather_d<128, false>(pl, k_src, v_src, k_pool, v_pool, mode, st);
+    return il ? launch_gather_d<64, true>(pl, k_src, v_src, k_pool, v_pool, mode, st)
+              : launch_gather_d<64, false>(pl, k_src, v_src, k_pool, v_pool, mode, st);
 }
 
 cudaError_t launch_rope_fresh(const tessera_plan *pl, void *q, void *k_new, cudaStream_t st) {
     if (pl->n_q == 0 || (!q && !k_new)) return cudaSuccess;
     const DeviceTables &d = pl->dev;
-    if (pl->cfg.head_dim == 128)
-        rope_fresh_kernel<128><<<(unsigned)pl->n_q, 128, 0, st>>>(static_cast<uint4 *>(q), static_cast<uint4 *>(k_new), d.q_pos,
-                                                                 d.inv_freq, pl->cfg.num_q_heads, pl->cfg.num_kv_heads);
-    else
-        rope_fresh_kernel<64><<<(unsigned)pl->n_q, 128, 0, st>>>(static_cast<uint4 *>(q), static_cast<uint4 *>(k_new), d.q_pos,
-                                                                d.inv_freq, pl->cfg.num_q_heads, pl->cfg.num_kv_heads);
+    auto *qp = static_cast<uint4 *>(q);
+    auto *kp = static_cast<uint4 *>(k_new);
+    const int Hq = pl->cfg.num_q_heads, Hkv = pl->cfg.num_kv_heads;
+    const unsigned n = (unsigned)pl->n_q;
+    const bool il = pl->cfg.rope_pairing == 1;
+    if (pl->cfg.head_dim == 128) {
+        if (il) rope_fresh_kernel<128, true><<<n, 128, 0, st>>>(qp, kp, d.q_pos, d.inv_freq, Hq, Hkv);
+        else rope_fresh_kernel<128, false><<<n, 128, 0, st>>>(qp, kp, d.q_pos, d.inv_freq, Hq, Hkv);
+    } else {
+        if (il) rope_fresh_kernel<64, true><<<n, 128, 0, st>>>(qp, kp, d.q_pos, d.inv_freq, Hq, Hkv);
+        else rope_fresh_kernel<64, false><<<n, 128, 0, st>>>(qp, kp, d.q_pos, d.inv_freq, Hq, Hkv);
+    }
     count_launch();
     return cudaGetLastError();
 }

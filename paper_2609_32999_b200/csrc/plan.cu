@@ -42,7 +42,8 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
     if (D != 64 && D != 128) return fail(TESSERA_UNSUPPORTED_SHAPE, fmt("head_dim %ld: only 64 and 128", D));
     if (B <= 0 || B % 8 != 0 || B > 128 || !is_pow2(B))
         return fail(TESSERA_UNSUPPORTED_SHAPE, fmt("page_size %ld: a power of two in 8..128", B));
-    if (cfg->rope_pairing != 0) return fail(TESSERA_UNSUPPORTED_SHAPE, "rope_pairing: only 0 (half-split pairs)");
+    if (cfg->rope_pairing != 0 && cfg->rope_pairing != 1)
+        return fail(TESSERA_UNSUPPORTED_SHAPE, "rope_pairing: 0 (half-split pairs) or 1 (interleaved pairs)");
     if (!cfg->inv_freq && !(cfg->rope_theta > 0.0)) return fail(TESSERA_INVALID_ARG, "rope_theta must be positive");
     if ((int64_t)num_pool_pages * B > (int64_t)INT32_MAX)
         return fail(TESSERA_UNSUPPORTED_SHAPE, "pool has more than 2^31 slots");

@@ -337,3 +337,28 @@ def test_rope_fresh_rotates_queries_and_keys_at_target_positions(make):
     zero = np.nonzero(w.recompute_pos == 0)[0]
     for j in zero:
         assert np.array_equal(q0[j], q1[j]) and np.array_equal(k0[j], k1[j])
+
+
+@pytest.mark.parametrize("shape", [wl.ModelShape(8, 2, 64, 16, 10000.0, rope_pairing=1),
+                                   wl.ModelShape(32, 8, 128, 64, 500000.0, rope_pairing=1)])
+def test_interleaved_rope_pairing(shape):
+    """Pairs (2m, 2m + 1) instead of (m, m + D/2): gather + shift, standalone shift and fresh rotation."""
+    w = wl.adversarial(seed=31, shape=shape)
+    _full_check(w)
+    _full_check(w, fuse=False)
+    dev = "cuda:0"
+    t = wl.make_tensors(w, device=dev, seed=45)
+    q0, k0 = orc.bf16_bits_to_f64(orc.bits(t.q)), orc.bf16_bits_to_f64(orc.bits(t.k_new))
+    tb.Plan(w).rope_fresh(t.q, t.k_new)
+    torch.cuda.synchronize()
+    q1, k1 = orc.bf16_bits_to_f64(orc.bits(t.q)), orc.bf16_bits_to_f64(orc.bits(t.k_new))
+    errs = []
+    for j in range(0, w.n_q, 3):
+        p = int(w.recompute_pos[j])
+        errs.append(np.abs(orc.rope_rotate(q0[j, 0], p, shape.rope_theta, pairing=1) - q1[j, 0]))
+        errs.append(np.abs(orc.rope_rotate(k0[j, 1], p, shape.rope_theta, pairing=1) - k1[j, 1]))
+    e = np.concatenate(errs)
+    assert e.max() <= gu.MAX_ABS and e.mean() <= gu.MEAN_ABS
+    # and it really differs from the half-split result
+    wrong = orc.rope_rotate(q0[5, 0], int(w.recompute_pos[5]), shape.rope_theta, pairing=0)
+    assert np.abs(wrong - q1[5, 0]).max() > 0.1 or int(w.recompute_pos[5]) == 0

@@ -92,7 +92,7 @@ def test_validation_errors():
     assert tb.plan_create_status(_mut(unit_cached_stride=st)) == tb.INVALID_ARG
     # shapes
     for bad in (wl.ModelShape(4, 3, 64, 16, 1e4), wl.ModelShape(4, 2, 96, 16, 1e4), wl.ModelShape(4, 2, 64, 12, 1e4),
-                wl.ModelShape(4, 2, 64, 16, 1e4, rope_pairing=1), wl.ModelShape(64, 2, 64, 16, 1e4)):
+                wl.ModelShape(4, 2, 64, 16, 1e4, rope_pairing=2), wl.ModelShape(64, 2, 64, 16, 1e4)):
         assert tb.plan_create_status(_mut(shape=bad)) == tb.UNSUPPORTED_SHAPE
     assert "page" in tb.last_error() or "head" in tb.last_error() or "group" in tb.last_error()
 
