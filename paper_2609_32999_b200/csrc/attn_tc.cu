@@ -22,7 +22,6 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
-#include <cstdio>
 
 #include "launch.h"
 #include "plan.h"
@@ -38,11 +37,7 @@ constexpr int kD = 128;            // head_dim
 constexpr int kPage = 64;          // page size
 constexpr int kStep = 128;         // keys per step (two pages)
 constexpr int kRows = 128;         // rows per query tile
-#ifdef TESSERA_ATTN_TRACE
-constexpr int kRing = 4;
-#else
 constexpr int kRing = 5;           // K/V ring slots
-#endif
 constexpr int kThreads = 384;        // 8 softmax warps, producer, MMA, 2 idle warps (register donors)
 
 constexpr uint32_t kQTileBytes = kRows * kD * 2;         // 32 KB: [d half][128 rows][128 B]
@@ -109,18 +104,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     __shared__ int s_abort;
     __shared__ float s_xchg[2][kRows];              // row maxima exchanged between the two column halves
     __shared__ int s_flag[2][2][4][2];              // [step parity][tile][warp pair][half]
-#ifdef TESSERA_ATTN_TRACE
-    __shared__ unsigned s_trace[2][16][8];
-    __shared__ unsigned s_ptrace[16][4];
-    __shared__ unsigned s_strace[2][16][4];
-#define STRACE(q, j, e) do { if ((j) >= 8 && (j) < 24) s_strace[q][(j) - 8][e] = (unsigned)clock64(); } while (0)
-#define TRACE(q, j, e) do { if ((j) >= 8 && (j) < 24) s_trace[q][(j) - 8][e] = (unsigned)clock64(); } while (0)
-#define PTRACE(j, e) do { if ((j) >= 8 && (j) < 24) s_ptrace[(j) - 8][e] = (unsigned)clock64(); } while (0)
-#else
-#define TRACE(q, j, e) do {} while (0)
-#define PTRACE(j, e) do {} while (0)
-#define STRACE(q, j, e) do {} while (0)
-#endif
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const AttnWork wk = work[blockIdx.x];
@@ -197,9 +180,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 #pragma unroll
                     for (int kv = 0; kv < 2; ++kv) {
                         const int item = 2 * j + kv, slot = item % kRing;
-                        PTRACE(j, 2 * kv);
                         mbar_wait(smem_u32(&bars.empty[slot]), ((item / kRing) & 1) ^ 1, abort_flag, status, 1 + kv);
-                        PTRACE(j, 2 * kv + 1);
                         const uint32_t fb = smem_u32(&bars.full[slot]);
                         mbar_expect_tx(fb, kSlotBytes);
                         const uint32_t dst = smem_u32(sm + kSmemRing + slot * kSlotBytes);
@@ -246,7 +227,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         if (lane == 0) issue_s(0);
         __syncwarp();
         for (int j = 0; j < n_steps; ++j) {
-            if (lane == 0 && q == 0) TRACE(0, j, 7);
             ring_wait(2 * j + 1, 5);                               // V_j
             const int vslot = (2 * j + 1) % kRing;
             const bool more = j + 1 < n_steps;
@@ -272,13 +252,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             }
             const bool next_s = j + 1 < my_steps;
             if (more) ring_wait(2 * j + 2, 3);                     // K_{j+1}
-            if (lane == 0 && q == 0) TRACE(1, j, 7);
             const uint32_t vbase = smem_u32(sm + kSmemRing + vslot * kSlotBytes);
-            if (lane == 0) TRACE(q, j, 4);
             mbar_wait(smem_u32(&bars.p_full[q]), j & 1, abort_flag, status, 6);
             tc_fence_after();
             if (lane == 0) {
-                TRACE(q, j, 5);
 #pragma unroll
                 for (int k = 0; k < kStep / 16; ++k) {
                     const uint64_t b = smem_desc_sw128(vbase + k * 2048, kHalfBytes, 1024);
@@ -288,7 +265,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 umma_commit(smem_u32(&bars.empty[vslot]));
                 if (next_s) issue_s(j + 1);
                 else if (more) mbar_arrive(smem_u32(&bars.empty[(2 * j + 2) % kRing]));
-                TRACE(q, j, 6);
             }
             __syncwarp();
         }
@@ -320,10 +296,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 if (q >= n_tiles || j >= (q ? n_steps1 : n_steps0)) continue;
                 const uint32_t tS = tmem + kTmemS + q * 128 + h * 64 + lane_base;
                 // S_j complete; this also means P.V of step j-1 has completed (it was issued earlier)
-                if (tid == 0) TRACE(q, j, 0);
                 mbar_wait(smem_u32(&bars.s_full[q]), j & 1, abort_flag, status, 7);
                 tc_fence_after();
-                if (tid == 0) TRACE(q, j, 1);
                 const int key0 = (step0 + j) * kStep + h * 64;
                 const bool masked = (step0 + j) * kStep + kStep > (q ? t1.kv_full : t0.kv_full);   // a causal limit falls in this step
                 const int pr = p_row[q];
@@ -337,7 +311,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     tmem_ld32(tS, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
                     tmem_ld32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
                     tmem_wait_ld();
-                    if (tid == 0) STRACE(q, j, 0);
                     if (masked) {
 #pragma unroll
                         for (int i = 0; i < 64; ++i)
@@ -375,14 +348,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     pass(false, true);
                     stale = !(sum <= 256.f);
                 }
-                if (tid == 0) STRACE(q, j, 1);
                 // both halves of a row must take the same decision
                 const int par = j & 1;
                 const bool warp_stale = __any_sync(0xffffffffu, stale);
                 if (lane == 0) s_flag[par][q][pair][h] = warp_stale ? 1 : 0;
                 named_sync(1 + pair, 64);
                 const bool redo = (s_flag[par][q][pair][0] | s_flag[par][q][pair][1]) != 0;
-                if (tid == 0) STRACE(q, j, 2);
                 float factor = 1.f;
                 if (redo) {
                     pass(true, false);
@@ -408,7 +379,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     }
                     pass(false, true);
                 }
-                if (tid == 0) TRACE(q, j, 2);
                 l_row[q] = l_row[q] * factor + sum;
                 // P as bf16 over the first 32 of this thread's 64 S columns
                 tmem_st16(tS, &pk[0]);
@@ -416,7 +386,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars.p_full[q]));
-                if (tid == 0) TRACE(q, j, 3);
             }
         }
 
@@ -480,20 +449,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
-#ifdef TESSERA_ATTN_TRACE
-    if (blockIdx.x == 0 && tid == 0) {
-        const unsigned t0 = s_trace[0][0][0];
-        for (int j = 0; j < 16; ++j) {
-            for (int qq = 0; qq < 2; ++qq)
-                printf("j %d q %d | sm: wait %u got %u exp %u arr %u | mma: wait %u got %u issued %u\n", j + 8, qq,
-                       s_trace[qq][j][0] - t0, s_trace[qq][j][1] - t0, s_trace[qq][j][2] - t0, s_trace[qq][j][3] - t0,
-                       s_trace[qq][j][4] - t0, s_trace[qq][j][5] - t0, s_trace[qq][j][6] - t0);
-            for (int qq = 0; qq < 2; ++qq) printf("   sm q%d: ld done %u compute done %u exchanged %u\n", qq, s_strace[qq][j][0] - t0, s_strace[qq][j][1] - t0, s_strace[qq][j][2] - t0);
-            printf("   mma ring: begin %u done %u | producer K: wait %u issue %u  V: wait %u issue %u\n", s_trace[0][j][7] - t0,
-                   s_trace[1][j][7] - t0, s_ptrace[j][0] - t0, s_ptrace[j][1] - t0, s_ptrace[j][2] - t0, s_ptrace[j][3] - t0);
-        }
-    }
-#endif
     if (warp == 9) tmem_dealloc(tmem, kTmemCols);
 }
 

@@ -8,6 +8,15 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def pytest_sessionstart(session):
+    """Build the CUDA library (nvcc cross-compiles without a GPU) and the C oracle when they are
+    missing or older than their sources, so that a fresh checkout can run the suite directly."""
+    from paper_2609_32999_b200 import build as lib_build
+    from oracle import tessera_oracle
+    lib_build.build()
+    tessera_oracle.build()
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on the B200 box)")
 
