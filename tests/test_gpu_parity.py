@@ -362,3 +362,17 @@ def test_interleaved_rope_pairing(shape):
     # and it really differs from the half-split result
     wrong = orc.rope_rotate(q0[5, 0], int(w.recompute_pos[5]), shape.rope_theta, pairing=0)
     assert np.abs(wrong - q1[5, 0]).max() > 0.1 or int(w.recompute_pos[5]) == 0
+
+
+@pytest.mark.parametrize("shape", [wl.ModelShape(4, 4, 64, 8, 10000.0), wl.ModelShape(16, 1, 64, 128, 10000.0),
+                                   wl.ModelShape(8, 4, 128, 32, 500000.0), wl.ModelShape(32, 8, 128, 64, 500000.0)])
+def test_degenerate_layouts(shape):
+    """One-token requests, one-token units, a unit that exactly fills a page, a request made of a single
+    recomputed token, page sizes 8 / 32 / 128 (generic kernel) and 64 (tensor-core kernel)."""
+    B = shape.page_size
+    reqs = [[1],                                                        # a single fresh token
+            [wl.unit(1, "one", cached_pos=3), 1],                       # one cached token + one fresh
+            [wl.unit(B, "page", recompute=(0,)), wl.unit(B, "page2", cached_pos=7, recompute=(B - 1,)), 1],
+            [2, wl.unit(2 * B + 1, "long", cached_pos=1, stride=0, recompute=(0, 2 * B)), 1]]
+    w = wl.build_workload("degenerate", shape, reqs, np.random.default_rng(3))
+    _full_check(w)
