@@ -453,35 +453,48 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 }
 
 // Merges the parts of a split-KV launch: for every row, O = sum_p O_p 2^(m_p - m) / sum_p l_p 2^(m_p - m)
-// with m = max_p m_p.  One block per (tile, KV head); a warp walks rows, lanes walk head_dim.
+// with m = max_p m_p.  One warp per row (lanes walk head_dim), 8 rows per block, kRows / 8 blocks per
+// (tile, KV head) item; all parts of a row are loaded before any is used.
 __global__ void __launch_bounds__(256)
 attn_combine_kernel(const CombineItem *__restrict__ items, const AttnTile *__restrict__ tiles,
                     const float *__restrict__ ws_o, const float2 *__restrict__ ws_ml, __nv_bfloat16 *__restrict__ out,
                     float *__restrict__ lse, int H_q, int H_kv, int g, int max_parts) {
-    const CombineItem it = items[blockIdx.x];
+    constexpr int kBlocksPerItem = kRows / 8;
+    const CombineItem it = items[blockIdx.x / kBlocksPerItem];
     const AttnTile t = tiles[it.tile];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = (blockIdx.x % kBlocksPerItem) * 8 + warp;
+    if (row >= t.n_tok * g) return;
     const size_t slot0 = ((size_t)it.tile * H_kv + it.kvh) * max_parts;
-    for (int row = warp; row < t.n_tok * g; row += 8) {
-        float m = -INFINITY;
-        for (int p = 0; p < it.n_parts; ++p) m = fmaxf(m, ws_ml[(slot0 + p) * kRows + row].x);
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        float l = 0.f;
-        for (int p = 0; p < it.n_parts; ++p) {
-            const float2 ml = ws_ml[(slot0 + p) * kRows + row];
-            const float w = exp2f(ml.x - m);
-            l += ml.y * w;
-            const float4 o = *reinterpret_cast<const float4 *>(ws_o + ((slot0 + p) * kRows + row) * kD + lane * 4);
-            acc.x = fmaf(o.x, w, acc.x); acc.y = fmaf(o.y, w, acc.y); acc.z = fmaf(o.z, w, acc.z); acc.w = fmaf(o.w, w, acc.w);
+    float2 ml[kSplitMaxParts];
+    float4 o[kSplitMaxParts];
+#pragma unroll
+    for (int p = 0; p < kSplitMaxParts; ++p)
+        if (p < it.n_parts) {
+            ml[p] = ws_ml[(slot0 + p) * kRows + row];
+            o[p] = *reinterpret_cast<const float4 *>(ws_o + ((slot0 + p) * kRows + row) * kD + lane * 4);
         }
-        const float inv = 1.f / l;
-        const int tok = t.q_begin + row / g, head = it.kvh * g + row % g;
-        uint2 pk;
-        pk.x = pack_bf16(acc.x * inv, acc.y * inv);
-        pk.y = pack_bf16(acc.z * inv, acc.w * inv);
-        *reinterpret_cast<uint2 *>(out + ((size_t)tok * H_q + head) * kD + lane * 4) = pk;
-        if (lse && lane == 0) lse[(size_t)tok * H_q + head] = (m + log2f(l)) * 0.6931471805599453f;
-    }
+    float m = -INFINITY;
+#pragma unroll
+    for (int p = 0; p < kSplitMaxParts; ++p)
+        if (p < it.n_parts) m = fmaxf(m, ml[p].x);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float l = 0.f;
+#pragma unroll
+    for (int p = 0; p < kSplitMaxParts; ++p)
+        if (p < it.n_parts) {
+            const float w = exp2f(ml[p].x - m);
+            l += ml[p].y * w;
+            acc.x = fmaf(o[p].x, w, acc.x); acc.y = fmaf(o[p].y, w, acc.y);
+            acc.z = fmaf(o[p].z, w, acc.z); acc.w = fmaf(o[p].w, w, acc.w);
+        }
+    const float inv = 1.f / l;
+    const int tok = t.q_begin + row / g, head = it.kvh * g + row % g;
+    uint2 pk;
+    pk.x = pack_bf16(acc.x * inv, acc.y * inv);
+    pk.y = pack_bf16(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2 *>(out + ((size_t)tok * H_q + head) * kD + lane * 4) = pk;
+    if (lse && lane == 0) lse[(size_t)tok * H_q + head] = (m + log2f(l)) * 0.6931471805599453f;
 }
 
 }  // namespace
@@ -515,7 +528,7 @@ cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, c
         const int c0 = chunk < 0 ? 0 : pl->chunk_combine_off[chunk];
         const int c1 = chunk < 0 ? (int)pl->combine.size() : pl->chunk_combine_off[chunk + 1];
         if (c1 > c0) {
-            attn_combine_kernel<<<c1 - c0, 256, 0, st>>>(d.combine + c0, d.tiles, d.ws_o, d.ws_ml, static_cast<__nv_bfloat16 *>(out),
+            attn_combine_kernel<<<(c1 - c0) * (kRows / 8), 256, 0, st>>>(d.combine + c0, d.tiles, d.ws_o, d.ws_ml, static_cast<__nv_bfloat16 *>(out),
                                                           lse, Hq, Hkv, g, pl->max_parts);
             count_launch();
         }

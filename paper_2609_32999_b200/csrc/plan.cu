@@ -197,6 +197,14 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
     auto row_of = [&](int64_t delta) {
         return (int32_t)(std::lower_bound(deltas.begin(), deltas.end(), delta) - deltas.begin());
     };
+    // Rows per gather block: 32, fewer when the batch is so small that the grid would not fill the GPU.
+    int item_tokens = kGatherItemTokens;
+    {
+        int64_t cached = 0;
+        for (int u = 0; u < n_units; ++u)
+            if (d->unit_page_off[u + 1] > d->unit_page_off[u]) cached += d->unit_len[u];
+        while (item_tokens > 8 && cached / item_tokens < 4 * 148) item_tokens /= 2;
+    }
     pl->cached_tokens = 0;
     for (int r = 0; r < batch; ++r)
         for (int u = d->unit_off[r]; u < d->unit_off[r + 1]; ++u) {
@@ -205,8 +213,8 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
             const int64_t d0 = (int64_t)tp - d->unit_cached_pos[u];
             const int step = (d->unit_target_stride ? d->unit_target_stride[u] : 1) - d->unit_cached_stride[u];
             const int32_t row0 = row_of(d0);       // step +-1: consecutive integers are consecutive rows
-            for (int i0 = 0; i0 < len; i0 += kGatherItemTokens) {
-                const int cnt = std::min(kGatherItemTokens, len - i0);
+            for (int i0 = 0; i0 < len; i0 += item_tokens) {
+                const int cnt = std::min(item_tokens, len - i0);
                 pl->items.push_back({(int32_t)pl->g_src.size(), cnt, row0 + i0 * step, step});
                 for (int i = i0; i < i0 + cnt; ++i) {
                     const int p = tp + i;
@@ -255,7 +263,7 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
         if (!pairs.empty() && (int)pairs.size() * Hkv < kSplitTargetBlocks) {
             int longest = 1;
             for (auto &pr : pairs) longest = std::max(longest, steps_of(pr.second >= 0 ? pr.second : pr.first));
-            const int want = (kSplitTargetBlocks + (int)pairs.size() * Hkv - 1) / ((int)pairs.size() * Hkv);
+            const int want = kSplitTargetBlocks / ((int)pairs.size() * Hkv);     // stay within one wave of blocks
             pl->max_parts = std::max(1, std::min({want, kSplitMaxParts, longest / kSplitMinSteps}));
         }
         pl->combine.clear();
