@@ -191,6 +191,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle attention sampling")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay each layer's launches from a captured CUDA graph (latency-bound small batches)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -211,7 +213,10 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     w = rank_workload(args.config, rank, args.requests)
+    t_plan = time.perf_counter()
     plan = tb.Plan(w)
+    torch.cuda.synchronize()
+    plan_create_ms = (time.perf_counter() - t_plan) * 1e3      # host placement + table upload, once per batch
     info = plan.info
     layers = [wl.make_tensors(w, layer=l, device=dev, seed=wl.BASE_SEED + rank) for l in range(args.layers)]
     sh = w.shape
@@ -229,6 +234,34 @@ def main():
         plan.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, out, lse)
         if ev is not None:
             ev[2].record(stream)
+
+    graphs = None
+    if args.graph:
+        # one graph per layer pool: compose + scatter + attention (+ combine) replayed as one launch
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(args.layers):
+                step(i)                         # warm up outside capture (function attributes, descriptors)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graphs = []
+        for i in range(args.layers):
+            gph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gph):
+                t = layers[i]
+                plan.kv_compose(t.k_pool, t.v_pool, fuse_rope=True)
+                plan.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, out, lse)
+            graphs.append(gph)
+        eager_step = step
+
+        def step(i, ev=None):                   # noqa: F811  (graph replay has no inner events)
+            if ev is not None:
+                ev[0].record(stream)
+            graphs[i % args.layers].replay()
+            if ev is not None:
+                ev[1].record(stream)
+                ev[2].record(stream)
 
     def barrier():
         torch.cuda.synchronize()
@@ -298,7 +331,8 @@ def main():
                    "head_dim": sh.head_dim, "page_size": sh.page_size,
                    "l2": "inputs larger than L2: %d per-layer KV pools of %.2f GB cycled"
                          % (args.layers, 2 * t0.k_pool.numel() * 2 / 1e9),
-                   "attn_kernel": "tcgen05" if info.attn_kernel == 1 else "simt"},
+                   "attn_kernel": "tcgen05" if info.attn_kernel == 1 else "simt",
+                   "cuda_graph": bool(args.graph)},
         "clocks": clocks,
         "gpu_launches": launches,
         "e2e": {"value": all_tokens / (e2e_ms_max / 1e3), "unit": UNIT,
@@ -319,6 +353,7 @@ def main():
                             "ms_per_launch": gather_ms, "bytes_per_launch": int(info.gather_bytes),
                             "traffic": NCU_TRAFFIC_PER_REQUEST_C4["gather"] * w.batch if args.config == 4 else None},
         "recompute_tokens_per_s": w.n_q * world / (ms_per_step / 1e3),
+        "plan_create_ms": plan_create_ms,
     }
     if not args.no_cpu_baseline:
         s = oracle_sample(w, host_bits(t0), args.cpu_budget)
