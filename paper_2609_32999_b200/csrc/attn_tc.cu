@@ -3,7 +3,7 @@
 //
 // One thread block works on one KV head and up to TWO query tiles of the same request (128 rows
 // each: 128/g recompute tokens x the g query heads of the group), which share every K/V page they
-// read.  A step covers 128 keys (two pages).  Warp roles (384 threads):
+// read.  A step covers 128 keys (1, 2, 4 or 8 pages of 128, 64, 32 or 16 tokens).  Warp roles (384 threads):
 //   warps 0-7  : softmax.  All eight work on one tile at a time and alternate between the tiles;
 //                warps 0-3 own columns 0-63 of a row, warps 4-7 columns 64-127 (TMEM lane = row)
 //   warp 8     : TMA producer - Q tiles once, then K and V of every step through one ring of
@@ -34,7 +34,6 @@ namespace {
 using namespace ptx;
 
 constexpr int kD = 128;            // head_dim
-constexpr int kPage = 64;          // page size
 constexpr int kStep = 128;         // keys per step (two pages)
 constexpr int kRows = 128;         // rows per query tile
 constexpr int kRing = 5;           // K/V ring slots
@@ -43,7 +42,6 @@ constexpr int kThreads = 384;        // 8 softmax warps, producer, MMA, 2 idle w
 constexpr uint32_t kQTileBytes = kRows * kD * 2;         // 32 KB: [d half][128 rows][128 B]
 constexpr uint32_t kSlotBytes = kStep * kD * 2;          // 32 KB: [d half][128 keys][128 B]
 constexpr uint32_t kHalfBytes = kSlotBytes / 2;          // 16 KB
-constexpr uint32_t kPageHalfBytes = kPage * 128;         // 8 KB: one page inside a d half
 constexpr uint32_t kSmemQ = 0;
 constexpr uint32_t kSmemRing = kSmemQ + 2 * kQTileBytes;
 constexpr uint32_t kSmemTotal = kSmemRing + kRing * kSlotBytes;
@@ -95,7 +93,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                const AttnWork *__restrict__ work, const int32_t *__restrict__ q_pos,
                const int32_t *__restrict__ page_off, const int32_t *__restrict__ pages,
                const int32_t *__restrict__ seq_len, __nv_bfloat16 *__restrict__ out, float *__restrict__ lse,
-               int H_q, int g, int H_kv, int num_pool_pages, float scale_log2, int max_parts,
+               int H_q, int g, int H_kv, int page_size, int num_pool_pages, float scale_log2, int max_parts,
                float *__restrict__ ws_o, float2 *__restrict__ ws_ml, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -118,7 +116,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const int n_steps1 = n_tiles == 2 ? min(wk.step_end, (t1.kv_len + kStep - 1) / kStep) - step0 : 0;
     const int n_steps = max(n_steps0, n_steps1);
     const int T = seq_len[t0.req];
-    const int req_pages = (T + kPage - 1) / kPage;
+    const int req_pages = (T + page_size - 1) / page_size;
+    const int pps = kStep / page_size;                 // pages per step: 1, 2, 4 or 8
     const int32_t *bt = pages + page_off[t0.req];
 
     if (tid == 0) {
@@ -166,15 +165,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             }
         }
         // ring item 2j = K of step j, item 2j+1 = V of step j
-        for (int j0 = 0; j0 < n_steps; j0 += 16) {
-            // lane l holds the id of page (2 * j0 + l); a page past the request's last one is fetched
-            // from outside the pool, which TMA fills with zeros
-            const int pi = 2 * (step0 + j0) + lane;
+        const int steps_per_fetch = 32 / pps;
+        const uint32_t page_bytes = (uint32_t)page_size * 128;     // one page inside a d half
+        for (int j0 = 0; j0 < n_steps; j0 += steps_per_fetch) {
+            // lane l holds the id of page (pps * (step0 + j0) + l); a page past the request's last one
+            // is fetched from outside the pool, which TMA fills with zeros
+            const int pi = pps * (step0 + j0) + lane;
             const int my_page = pi < req_pages ? bt[pi] : num_pool_pages;
-            const int jn = min(16, n_steps - j0);
+            const int jn = min(steps_per_fetch, n_steps - j0);
             for (int jj = 0; jj < jn; ++jj) {
-                const int pg0 = __shfl_sync(0xffffffffu, my_page, 2 * jj);
-                const int pg1 = __shfl_sync(0xffffffffu, my_page, 2 * jj + 1);
+                int pg[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) pg[k] = __shfl_sync(0xffffffffu, my_page, (pps * jj + k) & 31);
                 if (lane == 0) {
                     const int j = j0 + jj;
 #pragma unroll
@@ -185,10 +187,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                         mbar_expect_tx(fb, kSlotBytes);
                         const uint32_t dst = smem_u32(sm + kSmemRing + slot * kSlotBytes);
                         const CUtensorMap *tm = kv ? &tmap_v : &tmap_k;
-                        tma_load_4d(dst, tm, fb, 0, kvh, 0, pg0);
-                        tma_load_4d(dst + kPageHalfBytes, tm, fb, 0, kvh, 0, pg1);
-                        tma_load_4d(dst + kHalfBytes, tm, fb, 64, kvh, 0, pg0);
-                        tma_load_4d(dst + kHalfBytes + kPageHalfBytes, tm, fb, 64, kvh, 0, pg1);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k)
+                            if (k < pps) {
+                                tma_load_4d(dst + k * page_bytes, tm, fb, 0, kvh, 0, pg[k]);
+                                tma_load_4d(dst + kHalfBytes + k * page_bytes, tm, fb, 64, kvh, 0, pg[k]);
+                            }
                     }
                 }
                 __syncwarp();
@@ -506,14 +510,15 @@ cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, c
     const size_t n_work = chunk < 0 ? pl->work.size() : (size_t)(pl->chunk_work_off[chunk + 1] - pl->chunk_work_off[chunk]);
     if (n_work == 0) return cudaSuccess;
     const int Hq = pl->cfg.num_q_heads, Hkv = pl->cfg.num_kv_heads, g = Hq / Hkv;
-    if (pl->cfg.head_dim != kD || pl->cfg.page_size != kPage || kRows % g != 0) {
+    const int ps = pl->cfg.page_size;
+    if (pl->cfg.head_dim != kD || (ps != 16 && ps != 32 && ps != 64 && ps != 128) || kRows % g != 0) {
         *err = "shape outside the tcgen05 kernel's range";
         return cudaErrorNotSupported;
     }
     CUtensorMap tq, tk, tv;
     if (!make_q_tmap(&tq, q, pl->n_q, Hq, kD, g, kRows / g, err)) return cudaErrorInvalidValue;
-    if (!make_pool_tmap(&tk, k_pool, pl->num_pool_pages, kPage, Hkv, kD, err)) return cudaErrorInvalidValue;
-    if (!make_pool_tmap(&tv, v_pool, pl->num_pool_pages, kPage, Hkv, kD, err)) return cudaErrorInvalidValue;
+    if (!make_pool_tmap(&tk, k_pool, pl->num_pool_pages, ps, Hkv, kD, err)) return cudaErrorInvalidValue;
+    if (!make_pool_tmap(&tv, v_pool, pl->num_pool_pages, ps, Hkv, kD, err)) return cudaErrorInvalidValue;
     {
         cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemAlloc);
         if (e != cudaSuccess) { *err = "cudaFuncSetAttribute(shared memory)"; return e; }
@@ -522,7 +527,7 @@ cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, c
     const float scale_log2 = pl->sm_scale * 1.4426950408889634f;
     attn_tc_kernel<<<(unsigned)n_work, kThreads, kSmemAlloc, st>>>(
         tq, tk, tv, d.tiles, work, d.q_pos, d.page_off, d.pages, d.seq_len,
-        static_cast<__nv_bfloat16 *>(out), lse, Hq, g, Hkv, pl->num_pool_pages, scale_log2, pl->max_parts, d.ws_o, d.ws_ml, d.status);
+        static_cast<__nv_bfloat16 *>(out), lse, Hq, g, Hkv, ps, pl->num_pool_pages, scale_log2, pl->max_parts, d.ws_o, d.ws_ml, d.status);
     count_launch();
     if (pl->max_parts > 1) {
         const int c0 = chunk < 0 ? 0 : pl->chunk_combine_off[chunk];

@@ -391,3 +391,14 @@ def test_sharp_softmax_with_frequent_reference_refresh():
     # against the unrounded oracle keys the logits themselves move by up to |q| * 2^-9 * sqrt(D) here, so only
     # the kernel-alone comparison is meaningful at the tolerance; also check LSE finite and outputs normalised
     assert np.isfinite(g.lse_f).all() and np.abs(g.out_f).max() < 8.0
+
+
+@pytest.mark.parametrize("page", [16, 32, 128])
+def test_tensor_core_path_with_other_page_sizes(page):
+    """A 128-key step is 8, 4 or 1 pages instead of 2."""
+    shape = wl.ModelShape(32, 8, 128, page, 500000.0)
+    g, _ = _full_check(wl.adversarial(seed=40 + page, shape=shape))
+    assert g.plan.info.attn_kernel == 1
+    w = wl.build_workload("long", shape, [[9, wl.unit(900, "a", recompute=(0, 1, 450)), wl.unit(333, "b", cached_pos=4), 17],
+                                          [wl.unit(333, "b", cached_pos=4, recompute=(5,)), 3]], np.random.default_rng(page))
+    _full_check(w)
