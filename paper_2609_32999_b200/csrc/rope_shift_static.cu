@@ -1,8 +1,8 @@
 // tessera_rope_shift_static: the in-place RoPE shift for callers that may not allocate device
 // memory.  The regular path keeps its cos/sin table in memory that tessera_plan_create obtains with
-// cudaMalloc; code running inside a memory-pool-owning serving engine, inside a region where the
-// allocator is frozen (for instance while a stream is being captured), or under a strict
-// no-allocation policy after start-up cannot do that.  Here the table lives in a fixed array that is
+// cudaMalloc; code running inside a memory-pool-owning serving engine, in a phase where the
+// allocator must stay untouched, or under a strict no-allocation policy after start-up cannot do
+// that.  Here the table lives in a fixed array that is
 // part of the library image, so a call allocates nothing - neither through cudaMalloc nor through
 // any allocating library routine.
 #include <cmath>
@@ -102,7 +102,7 @@ extern "C" int32_t tessera_rope_shift_static(const tessera_model_cfg *cfg, void 
     float2 *table = g_scratch_addr[dev];
 
     // cos/sin in fp64, one rounding to fp32 - the same numbers the plan-based path tabulates.
-    static thread_local float host_table[kMaxShifts * kMaxHalf * 2];
+    std::vector<float> host_table((size_t)n_shifts * (D / 2) * 2);   // host memory only; staged by the copy below
     for (int r = 0; r < n_shifts; ++r)
         for (int m = 0; m < D / 2; ++m) {
             const double w = cfg->inv_freq ? cfg->inv_freq[m] : std::pow(cfg->rope_theta, -2.0 * m / D);
@@ -111,7 +111,7 @@ extern "C" int32_t tessera_rope_shift_static(const tessera_model_cfg *cfg, void 
             host_table[(r * (D / 2) + m) * 2 + 1] = (float)std::sin(ang);
         }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    e = cudaMemcpyAsync(table, host_table, (size_t)n_shifts * (D / 2) * sizeof(float2), cudaMemcpyHostToDevice, st);
+    e = cudaMemcpyAsync(table, host_table.data(), (size_t)n_shifts * (D / 2) * sizeof(float2), cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess)
         return api_set_error(TESSERA_CUDA_ERROR, std::string("rope_shift_static: table upload: ") + cudaGetErrorString(e));
     const int blocks = (n_slots + 7) / 8;
