@@ -122,10 +122,9 @@ def check_untouched(g):
     assert np.array_equal(g.v_after[mask], g.v_before[mask]), "a non-destination V page changed"
 
 
-def check_attention(g, asm, rows_by_request=None, use_pool_k=False):
-    """Attention outputs vs the oracle.  rows_by_request: {r: (row_q, row_h, row_pos)} or None for
-    every row.  use_pool_k: feed the oracle the bf16 keys the GPU actually left in its pages (the
-    attention kernel alone) instead of its own unrounded fp64 keys (the whole path)."""
+def check_attention(g, asm, rows_by_request=None):
+    """Attention outputs of the whole path vs the oracle, which attends over its own unrounded fp64
+    keys.  rows_by_request: {r: (row_q, row_h, row_pos)} or None for every row."""
     w = g.w
     sh = w.shape
     row = sh.num_kv_heads * sh.head_dim
@@ -138,9 +137,6 @@ def check_attention(g, asm, rows_by_request=None, use_pool_k=False):
         if len(jj) == 0:
             continue
         k = a.k
-        if use_pool_k:
-            slots = dest_slots(g, r)
-            k = orc.bf16_bits_to_f64(g.k_after.reshape(-1, row)[slots]).reshape(a.k.shape)
         o, l = orc.attention_rows(w, k, a.v_bits, g.q_bits, jj, hh, pp)
         all_err.append(np.abs(g.out_f[jj, hh] - o).ravel())
         if g.lse_f is not None:
@@ -168,3 +164,68 @@ def sample_rows(w, r, rng, n_random, tile_tokens):
         rh = rng.integers(0, H, size=n_random).astype(np.int32)
         jj, hh = np.concatenate([jj, rj]), np.concatenate([hh, rh])
     return jj, hh, w.recompute_pos[jj].astype(np.int32)
+
+
+def host_assembled_pools(w, t):
+    """The state of the pools after gather + shift + scatter as the ORACLE computes it, with rotated keys
+    rounded to bf16 on the host: destination pages filled from oracle.assemble, everything else left
+    as generated.  Returns (k_pool, v_pool) device tensors and {request: fp64 K actually stored}."""
+    sh = w.shape
+    row = sh.num_kv_heads * sh.head_dim
+    kb, vb, knb, vnb = (orc.bits(x) for x in (t.k_pool, t.v_pool, t.k_new, t.v_new))
+    st, page_off, pages, _, _ = orc.placement(w)
+    assert st == 0
+    k_img, v_img = kb.copy().reshape(-1, row), vb.copy().reshape(-1, row)
+    stored = {}
+    B = sh.page_size
+    for r in range(w.batch):
+        a = orc.assemble(w, r, kb, vb, knb, vnb)
+        T = int(w.seq_len[r])
+        if T == 0:
+            continue
+        p = np.arange(T)
+        slots = pages[page_off[r] + p // B].astype(np.int64) * B + p % B
+        k_round = torch.from_numpy(a.k.reshape(T, row)).to(torch.bfloat16)          # one rounding, on the host
+        k_bits = k_round.view(torch.int16).numpy().view(np.uint16).copy()
+        ex = a.k_exact != 0
+        k_bits[ex] = a.k_bits.reshape(T, row)[ex]                                    # bit copies stay bit copies
+        k_img[slots] = k_bits
+        v_img[slots] = a.v_bits.reshape(T, row)
+        stored[r] = (orc.bf16_bits_to_f64(k_bits).reshape(a.k.shape), a.v_bits)
+    dev = t.k_pool.device
+    to_dev = lambda img: torch.from_numpy(img.view(np.int16).reshape(kb.shape)).view(torch.bfloat16).to(dev)
+    return to_dev(k_img), to_dev(v_img), stored
+
+
+def check_attention_alone(w, seed=None, layer=0):
+    """The attention kernel by itself: pages assembled by the oracle on the host (rotated keys rounded
+    once to bf16), attention on the GPU without any gather or scatter, compared with the oracle
+    attending over exactly those stored keys."""
+    dev = "cuda:0"
+    t = wl.make_tensors(w, layer=layer, device=dev, seed=seed)
+    k_pool, v_pool, stored = host_assembled_pools(w, t)
+    plan = tb.Plan(w)
+    sh = w.shape
+    out = torch.zeros(w.n_q, sh.num_q_heads, sh.head_dim, dtype=torch.bfloat16, device=dev)
+    lse = torch.zeros(w.n_q, sh.num_q_heads, dtype=torch.float32, device=dev)
+    plan.partial_prefill_attn(k_pool, v_pool, t.q, None, None, out, lse)
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+    out_f = out.float().cpu().numpy().astype(np.float64)
+    lse_f = lse.cpu().numpy().astype(np.float64)
+    q_bits = orc.bits(t.q)
+    errs, lerr = [], []
+    for r, (k, v_bits) in stored.items():
+        jj, hh, pp = orc.request_rows(w, r)
+        if len(jj) == 0:
+            continue
+        o, l = orc.attention_rows(w, k, v_bits, q_bits, jj, hh, pp)
+        errs.append(np.abs(out_f[jj, hh] - o).ravel())
+        lerr.append(np.abs(lse_f[jj, hh] - l))
+    if not errs:
+        return 0.0, 0.0
+    e = np.concatenate(errs)
+    assert np.isfinite(e).all()
+    assert e.max() <= MAX_ABS and e.mean() <= MEAN_ABS, "attention alone: max %.4g mean %.4g" % (e.max(), e.mean())
+    assert np.concatenate(lerr).max() <= 5e-3, "attention alone: LSE max-abs %.4g" % np.concatenate(lerr).max()
+    return float(e.max()), float(e.mean())
