@@ -129,11 +129,11 @@ def host_bits(t):
     return tuple(orc.bits(x) for x in (t.k_pool, t.v_pool, t.q, t.k_new, t.v_new))
 
 
-def rank_workload(config: int, rank: int, requests=None):
+def rank_workload(config: int, rank: int, requests=None, policy=None):
     """Every rank owns an independent batch of the same configuration: requests never interact
     (no cross-request attention), so the path shards by request with no data-path collective."""
     from paper_2609_32999_b200 import workloads as wl
-    return wl.config(config, seed=wl.BASE_SEED + config + 7919 * rank, requests_override=requests)
+    return wl.config(config, seed=wl.BASE_SEED + config + 7919 * rank, requests_override=requests, policy=policy)
 
 
 def aggregate(times_ms, tokens, world: int, device: str):
@@ -155,7 +155,7 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2609_32999_b200 import workloads as wl
-    w = wl.config(args.config, requests_override=args.requests)
+    w = wl.config(args.config, requests_override=args.requests, policy=args.policy)
     t = wl.make_tensors(w, layer=0, device="cpu")
     bits = host_bits(t)
     per_step_budget = max(2.0, min(20.0, 90.0 / max(args.steps + args.warmup, 1)))
@@ -191,6 +191,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle attention sampling")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--policy", default=None, choices=["reuse", "lru", "lfu"],
+                    help="residency of the units decided by a cache policy instead of 'all cached' (configs 2-4)")
     ap.add_argument("--graph", action="store_true",
                     help="replay each layer's launches from a captured CUDA graph (latency-bound small batches)")
     args = ap.parse_args()
@@ -212,7 +214,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    w = rank_workload(args.config, rank, args.requests)
+    w = rank_workload(args.config, rank, args.requests, args.policy)
     t_plan = time.perf_counter()
     plan = tb.Plan(w)
     torch.cuda.synchronize()
@@ -332,7 +334,7 @@ def main():
                    "l2": "inputs larger than L2: %d per-layer KV pools of %.2f GB cycled"
                          % (args.layers, 2 * t0.k_pool.numel() * 2 / 1e9),
                    "attn_kernel": "tcgen05" if info.attn_kernel == 1 else "simt",
-                   "cuda_graph": bool(args.graph)},
+                   "cuda_graph": bool(args.graph), "residency": args.policy or "all units cached"},
         "clocks": clocks,
         "gpu_launches": launches,
         "e2e": {"value": all_tokens / (e2e_ms_max / 1e3), "unit": UNIT,

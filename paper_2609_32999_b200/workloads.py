@@ -175,8 +175,29 @@ def zipf_ranks(rng: np.random.Generator, n: int, pool: int, s: float, distinct: 
 LLAMA8B = dict(num_q_heads=32, num_kv_heads=8, head_dim=128, page_size=64, rope_theta=500000.0)
 
 
-def config(index: int, seed: Optional[int] = None, requests_override: Optional[int] = None) -> Workload:
+def _policy_cache(policy: Optional[str], capacity_blocks: int, avg_blocks_per_request: float):
+    """Residency model for configs 2-4: None = every unit is a hit (the configurations as stated);
+    "reuse" = the paper's score-based admission / eviction (Sec. 5.2), "lru", "lfu" = baselines."""
+    if policy is None:
+        return None
+    from . import residency as rs
+    if policy == "reuse":
+        return rs.ReuseScoreCache(capacity_blocks, rs.ReuseScoreCache.window_for(capacity_blocks, avg_blocks_per_request))
+    if policy == "lru":
+        return rs.LRUCache(capacity_blocks)
+    if policy == "lfu":
+        return rs.LFUCache(capacity_blocks)
+    raise ValueError("policy must be None, 'reuse', 'lru' or 'lfu'")
+
+
+def config(index: int, seed: Optional[int] = None, requests_override: Optional[int] = None,
+           policy: Optional[str] = None, warm_requests: int = 400, capacity_fraction: float = 0.1) -> Workload:
     """The five benchmark configurations, index 1..5.
+
+    With `policy` (configs 2-4) residency is no longer "everything cached": a cache holding
+    `capacity_fraction` of the unit pool is warmed with `warm_requests` requests of the same
+    popularity law, and the batch's units are hits only if resident; the others are uncached and
+    fully recomputed (Sec. 5.3 "Preparation failures": computed from text).
 
     `requests_override` shrinks (or grows) the number of requests of the batched
     configurations (3, 4, 5) while keeping every per-request rule; it is how the
@@ -190,20 +211,29 @@ def config(index: int, seed: Optional[int] = None, requests_override: Optional[i
         return build_workload("c1-tiny", shape, [segs], rng)
     if index == 2:
         shape = ModelShape(**LLAMA8B)
+        cache = _policy_cache(policy, int(capacity_fraction * 1000 * 8), 10 * 8)
+        for _ in range(warm_requests if cache else 0):
+            cache.request([(k, 8) for k in zipf_ranks(rng, 10, 1000, 1.0, distinct=True)])
         ranks = zipf_ranks(rng, 10, 1000, 1.0, distinct=True)
-        segs = [64] + [_UnitSpec(("c", k), 512, recompute=range(16)) for k in ranks] + [128]
+        hits = cache.request([(k, 8) for k in ranks]) if cache else [True] * 10
+        segs = [64] + [_UnitSpec(("c", k), 512, cached=h, recompute=range(16)) for k, h in zip(ranks, hits)] + [128]
         return build_workload("c2-rag-single", shape, [segs], rng)
     if index == 3:
         shape = ModelShape(**LLAMA8B)
         nreq = requests_override or 16
         rec_len = rng.integers(128, 385, size=5000)      # length fixed per pool id
         id_perm = rng.permutation(5000)
+        blocks_of = lambda i: -(-int(rec_len[i]) // 64)
+        cache = _policy_cache(policy, int(capacity_fraction * sum(blocks_of(i) for i in range(5000))), 20 * 4.5)
+        for _ in range(warm_requests if cache else 0):
+            cache.request([(int(id_perm[k - 1]), blocks_of(int(id_perm[k - 1]))) for k in zipf_ranks(rng, 20, 5000, 1.1, distinct=True)])
         reqs = []
         for _ in range(nreq):
             ranks = zipf_ranks(rng, 20, 5000, 1.1, distinct=True)
             ids = [int(id_perm[k - 1]) for k in ranks]
+            hits = cache.request([(i, blocks_of(i)) for i in ids]) if cache else [True] * 20
             order = rng.permutation(20)
-            segs = [256] + [_UnitSpec(("m", ids[o]), int(rec_len[ids[o]]), recompute=range(8))
+            segs = [256] + [_UnitSpec(("m", ids[o]), int(rec_len[ids[o]]), cached=hits[o], recompute=range(8))
                             for o in order] + [96]
             reqs.append(segs)
         return build_workload("c3-agent-memory", shape, reqs, rng)
@@ -211,10 +241,14 @@ def config(index: int, seed: Optional[int] = None, requests_override: Optional[i
         shape = ModelShape(**LLAMA8B)
         nreq = requests_override or 4
         id_perm = rng.permutation(4000)
+        cache = _policy_cache(policy, int(capacity_fraction * 4000 * 8), 64 * 8)
+        for _ in range(warm_requests if cache else 0):
+            cache.request([(int(id_perm[k - 1]), 8) for k in zipf_ranks(rng, 64, 4000, 0.9, distinct=True)])
         reqs = []
         for _ in range(nreq):
             ranks = zipf_ranks(rng, 64, 4000, 0.9, distinct=True)
-            segs = [_UnitSpec(("c", int(id_perm[k - 1])), 512, recompute=range(32)) for k in ranks] + [256]
+            hits = cache.request([(int(id_perm[k - 1]), 8) for k in ranks]) if cache else [True] * 64
+            segs = [_UnitSpec(("c", int(id_perm[k - 1])), 512, cached=h, recompute=range(32)) for k, h in zip(ranks, hits)] + [256]
             reqs.append(segs)
         return build_workload("c4-long-rag", shape, reqs, rng, n_layers=32)
     if index == 5:

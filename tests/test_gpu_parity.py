@@ -423,3 +423,10 @@ def test_tensor_core_path_with_other_page_sizes(page):
     w = wl.build_workload("long", shape, [[9, wl.unit(900, "a", recompute=(0, 1, 450)), wl.unit(333, "b", cached_pos=4), 17],
                                           [wl.unit(333, "b", cached_pos=4, recompute=(5,)), 3]], np.random.default_rng(page))
     _full_check(w)
+
+
+def test_residency_decided_by_the_reuse_score_policy():
+    """Config 3 with hits and misses chosen by the score-based admission rule: missed records are
+    recomputed in full inside the same extend pass."""
+    w = wl.config(3, requests_override=3, policy="reuse")
+    _full_check(w)
