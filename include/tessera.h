@@ -18,6 +18,9 @@
  *     only the opaque plan (its host tables, device tables and staging buffers).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Device
  *     work is enqueued on it and the call returns without waiting, unless stated otherwise.
+ *   - One plan serves every layer of its batch, one call after the other.  Calls on the SAME plan
+ *     must not overlap on the GPU (two streams without ordering): a plan owns one status word, one
+ *     split-KV workspace and one set of staging buffers.  Different plans are independent.
  *   - All K/V/Q/O tensors are bf16 (2 bytes, raw bits), indices are int32.
  *   - KV pool layout (one K pool and one V pool per layer, same page ids in every layer):
  *         [num_pool_pages][page_size][num_kv_heads][head_dim]   bf16, contiguous,
