@@ -33,19 +33,23 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kD = 128;            // head_dim
 constexpr int kStep = 128;         // keys per step (two pages)
 constexpr int kRows = 128;         // rows per query tile
 constexpr int kRing = 5;           // K/V ring slots
 constexpr int kThreads = 384;        // 8 softmax warps, producer, MMA, 2 idle warps (register donors)
 
-constexpr uint32_t kQTileBytes = kRows * kD * 2;         // 32 KB: [d half][128 rows][128 B]
-constexpr uint32_t kSlotBytes = kStep * kD * 2;          // 32 KB: [d half][128 keys][128 B]
-constexpr uint32_t kHalfBytes = kSlotBytes / 2;          // 16 KB
-constexpr uint32_t kSmemQ = 0;
-constexpr uint32_t kSmemRing = kSmemQ + 2 * kQTileBytes;
-constexpr uint32_t kSmemTotal = kSmemRing + kRing * kSlotBytes;
-constexpr uint32_t kSmemAlloc = kSmemTotal + 1024;       // slack for the 1024-byte alignment
+// Shared-memory geometry for head_dim D (64 or 128): a tile of 128 rows is stored as D/64 "halves" of
+// [128 rows][128 B] (64 elements per row, 128-byte swizzle).
+constexpr uint32_t kHalfBytes = 128 * 128;                                     // 16 KB
+template <int D> struct Geo {
+    static constexpr int kHalves = D / 64;
+    static constexpr uint32_t kQTileBytes = kHalves * kHalfBytes;              // Q tile: 16 / 32 KB
+    static constexpr uint32_t kSlotBytes = kHalves * kHalfBytes;               // K or V of one step
+    static constexpr uint32_t kSmemQ = 0;
+    static constexpr uint32_t kSmemRing = kSmemQ + 2 * kQTileBytes;
+    static constexpr uint32_t kSmemTotal = kSmemRing + kRing * kSlotBytes;
+    static constexpr uint32_t kSmemAlloc = kSmemTotal + 1024;                  // slack for the 1024-byte alignment
+};
 
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemS = 0;      // S[tile] at tile * 128 (P[tile] = its first 64 columns)
@@ -87,6 +91,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return r;
 }
 
+template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, const AttnTile *__restrict__ tiles,
@@ -97,6 +102,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                float *__restrict__ ws_o, float2 *__restrict__ ws_ml, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    using G = Geo<D>;
+    constexpr int kD = D;
+    constexpr uint32_t kQTileBytes = G::kQTileBytes, kSlotBytes = G::kSlotBytes;
+    constexpr uint32_t kSmemQ = G::kSmemQ, kSmemRing = G::kSmemRing;
+    constexpr int kOCols = D / 2;                      // accumulator columns per softmax thread (row, column half)
     __shared__ __align__(8) Barriers bars;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
@@ -160,8 +170,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 const AttnTile &t = q ? t1 : t0;
                 const uint32_t bar = smem_u32(&bars.q_full[q]);
                 mbar_expect_tx(bar, kQTileBytes);
-                tma_load_3d(smem_u32(sm + kSmemQ + q * kQTileBytes), &tmap_q, bar, 0, kvh * g, t.q_begin);
-                tma_load_3d(smem_u32(sm + kSmemQ + q * kQTileBytes + kQTileBytes / 2), &tmap_q, bar, 64, kvh * g, t.q_begin);
+#pragma unroll
+                for (int hf = 0; hf < G::kHalves; ++hf)
+                    tma_load_3d(smem_u32(sm + kSmemQ + q * kQTileBytes + hf * kHalfBytes), &tmap_q, bar, hf * 64, kvh * g, t.q_begin);
             }
         }
         // ring item 2j = K of step j, item 2j+1 = V of step j
@@ -190,8 +201,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 #pragma unroll
                         for (int k = 0; k < 8; ++k)
                             if (k < pps) {
-                                tma_load_4d(dst + k * page_bytes, tm, fb, 0, kvh, 0, pg[k]);
-                                tma_load_4d(dst + kHalfBytes + k * page_bytes, tm, fb, 64, kvh, 0, pg[k]);
+#pragma unroll
+                                for (int hf = 0; hf < G::kHalves; ++hf)
+                                    tma_load_4d(dst + hf * kHalfBytes + k * page_bytes, tm, fb, hf * 64, kvh, 0, pg[k]);
                             }
                     }
                 }
@@ -218,7 +230,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             const uint32_t kbase = smem_u32(sm + kSmemRing + ((2 * j) % kRing) * kSlotBytes);
 #pragma unroll
             for (int k = 0; k < kD / 16; ++k) {
-                const uint64_t a = smem_desc_sw128(qbase + (k / 4) * (kQTileBytes / 2) + (k % 4) * 32, 16, 1024);
+                const uint64_t a = smem_desc_sw128(qbase + (k / 4) * kHalfBytes + (k % 4) * 32, 16, 1024);
                 const uint64_t b = smem_desc_sw128(kbase + (k / 4) * kHalfBytes + (k % 4) * 32, 16, 1024);
                 umma_ss(tS, a, b, idesc_s, k > 0);
             }
@@ -250,7 +262,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 // issuing warps may write these zeros; the values agree.)
                 uint8_t *v = sm + kSmemRing + vslot * kSlotBytes;
                 for (int r = T - (step0 + j) * kStep; r < kStep; ++r)
-                    if (lane < 16) *reinterpret_cast<uint4 *>(v + (lane >> 3) * kHalfBytes + r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    if (lane < 8 * G::kHalves) *reinterpret_cast<uint4 *>(v + (lane >> 3) * kHalfBytes + r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
                 fence_proxy_async_smem();
                 __syncwarp();
             }
@@ -370,9 +382,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     }
                     named_sync(1 + pair, 64);          // s_xchg may be rewritten after this point
                     if (j > 0) {
-                        const uint32_t tO = tmem + kTmemO + q * 128 + h * 64 + lane_base;
+                        const uint32_t tO = tmem + kTmemO + q * 128 + h * kOCols + lane_base;
 #pragma unroll
-                        for (int c = 0; c < 2; ++c) {
+                        for (int c = 0; c < kOCols / 32; ++c) {
                             uint32_t o[32];
                             tmem_ld32(tO + c * 32, o);
                             tmem_wait_ld();
@@ -408,10 +420,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             if (wke.n_parts > 1) {
                 // split-KV part: unnormalised accumulator, reference maximum and sum go to the workspace
                 const size_t slot = ((size_t)(q ? wke.tile_b : wke.tile_a) * H_kv + kvh) * max_parts + wke.part;
-                float *po = ws_o + (slot * kRows + row) * kD + h * 64;
-                const uint32_t tOp = tmem + kTmemO + q * 128 + h * 64 + lane_base;
+                float *po = ws_o + (slot * kRows + row) * kD + h * kOCols;
+                const uint32_t tOp = tmem + kTmemO + q * 128 + h * kOCols + lane_base;
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
+                for (int c = 0; c < kOCols / 32; ++c) {
                     uint32_t o[32];
                     tmem_ld32(tOp + c * 32, o);
                     tmem_wait_ld();
@@ -424,10 +436,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             }
             const float inv = 1.f / l_tot;
             const int head = kvh * g + row % g;
-            __nv_bfloat16 *orow = out + ((size_t)(t.q_begin + tok[q]) * H_q + head) * kD + h * 64;
-            const uint32_t tO = tmem + kTmemO + q * 128 + h * 64 + lane_base;
+            __nv_bfloat16 *orow = out + ((size_t)(t.q_begin + tok[q]) * H_q + head) * kD + h * kOCols;
+            const uint32_t tO = tmem + kTmemO + q * 128 + h * kOCols + lane_base;
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < kOCols / 32; ++c) {
                 uint32_t o[32];
                 tmem_ld32(tO + c * 32, o);
                 tmem_wait_ld();
@@ -459,6 +471,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 // Merges the parts of a split-KV launch: for every row, O = sum_p O_p 2^(m_p - m) / sum_p l_p 2^(m_p - m)
 // with m = max_p m_p.  One warp per row (lanes walk head_dim), 8 rows per block, kRows / 8 blocks per
 // (tile, KV head) item; all parts of a row are loaded before any is used.
+template <int kD>
 __global__ void __launch_bounds__(256)
 attn_combine_kernel(const CombineItem *__restrict__ items, const AttnTile *__restrict__ tiles,
                     const float *__restrict__ ws_o, const float2 *__restrict__ ws_ml, __nv_bfloat16 *__restrict__ out,
@@ -476,7 +489,8 @@ attn_combine_kernel(const CombineItem *__restrict__ items, const AttnTile *__res
     for (int p = 0; p < kSplitMaxParts; ++p)
         if (p < it.n_parts) {
             ml[p] = ws_ml[(slot0 + p) * kRows + row];
-            o[p] = *reinterpret_cast<const float4 *>(ws_o + ((slot0 + p) * kRows + row) * kD + lane * 4);
+            o[p] = lane * 4 < kD ? *reinterpret_cast<const float4 *>(ws_o + ((slot0 + p) * kRows + row) * kD + lane * 4)
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     float m = -INFINITY;
 #pragma unroll
@@ -497,35 +511,28 @@ attn_combine_kernel(const CombineItem *__restrict__ items, const AttnTile *__res
     uint2 pk;
     pk.x = pack_bf16(acc.x * inv, acc.y * inv);
     pk.y = pack_bf16(acc.z * inv, acc.w * inv);
-    *reinterpret_cast<uint2 *>(out + ((size_t)tok * H_q + head) * kD + lane * 4) = pk;
+    if (lane * 4 < kD) *reinterpret_cast<uint2 *>(out + ((size_t)tok * H_q + head) * kD + lane * 4) = pk;
     if (lse && lane == 0) lse[(size_t)tok * H_q + head] = (m + log2f(l)) * 0.6931471805599453f;
 }
 
-}  // namespace
-
-cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
-                           float *lse, int chunk, cudaStream_t st, std::string *err) {
-    if (pl->n_q == 0 || pl->work.empty()) return cudaSuccess;
+template <int D>
+cudaError_t launch_attn_tc_d(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
+                             float *lse, int chunk, cudaStream_t st, std::string *err) {
     const AttnWork *work = chunk < 0 ? pl->dev.work : pl->dev.work_chunked + pl->chunk_work_off[chunk];
     const size_t n_work = chunk < 0 ? pl->work.size() : (size_t)(pl->chunk_work_off[chunk + 1] - pl->chunk_work_off[chunk]);
     if (n_work == 0) return cudaSuccess;
-    const int Hq = pl->cfg.num_q_heads, Hkv = pl->cfg.num_kv_heads, g = Hq / Hkv;
-    const int ps = pl->cfg.page_size;
-    if (pl->cfg.head_dim != kD || (ps != 16 && ps != 32 && ps != 64 && ps != 128) || kRows % g != 0) {
-        *err = "shape outside the tcgen05 kernel's range";
-        return cudaErrorNotSupported;
-    }
+    const int Hq = pl->cfg.num_q_heads, Hkv = pl->cfg.num_kv_heads, g = Hq / Hkv, ps = pl->cfg.page_size;
     CUtensorMap tq, tk, tv;
-    if (!make_q_tmap(&tq, q, pl->n_q, Hq, kD, g, kRows / g, err)) return cudaErrorInvalidValue;
-    if (!make_pool_tmap(&tk, k_pool, pl->num_pool_pages, ps, Hkv, kD, err)) return cudaErrorInvalidValue;
-    if (!make_pool_tmap(&tv, v_pool, pl->num_pool_pages, ps, Hkv, kD, err)) return cudaErrorInvalidValue;
+    if (!make_q_tmap(&tq, q, pl->n_q, Hq, D, g, kRows / g, err)) return cudaErrorInvalidValue;
+    if (!make_pool_tmap(&tk, k_pool, pl->num_pool_pages, ps, Hkv, D, err)) return cudaErrorInvalidValue;
+    if (!make_pool_tmap(&tv, v_pool, pl->num_pool_pages, ps, Hkv, D, err)) return cudaErrorInvalidValue;
     {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemAlloc);
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Geo<D>::kSmemAlloc);
         if (e != cudaSuccess) { *err = "cudaFuncSetAttribute(shared memory)"; return e; }
     }
     const DeviceTables &d = pl->dev;
     const float scale_log2 = pl->sm_scale * 1.4426950408889634f;
-    attn_tc_kernel<<<(unsigned)n_work, kThreads, kSmemAlloc, st>>>(
+    attn_tc_kernel<D><<<(unsigned)n_work, kThreads, Geo<D>::kSmemAlloc, st>>>(
         tq, tk, tv, d.tiles, work, d.q_pos, d.page_off, d.pages, d.seq_len,
         static_cast<__nv_bfloat16 *>(out), lse, Hq, g, Hkv, ps, pl->num_pool_pages, scale_log2, pl->max_parts, d.ws_o, d.ws_ml, d.status);
     count_launch();
@@ -533,14 +540,28 @@ cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, c
         const int c0 = chunk < 0 ? 0 : pl->chunk_combine_off[chunk];
         const int c1 = chunk < 0 ? (int)pl->combine.size() : pl->chunk_combine_off[chunk + 1];
         if (c1 > c0) {
-            attn_combine_kernel<<<(c1 - c0) * (kRows / 8), 256, 0, st>>>(d.combine + c0, d.tiles, d.ws_o, d.ws_ml, static_cast<__nv_bfloat16 *>(out),
-                                                          lse, Hq, Hkv, g, pl->max_parts);
+            attn_combine_kernel<D><<<(c1 - c0) * (kRows / 8), 256, 0, st>>>(d.combine + c0, d.tiles, d.ws_o, d.ws_ml, static_cast<__nv_bfloat16 *>(out),
+                                                                          lse, Hq, Hkv, g, pl->max_parts);
             count_launch();
         }
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) *err = "kernel launch";
     return e;
+}
+
+}  // namespace
+
+cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
+                           float *lse, int chunk, cudaStream_t st, std::string *err) {
+    if (pl->n_q == 0 || pl->work.empty()) return cudaSuccess;
+    const int D = pl->cfg.head_dim, ps = pl->cfg.page_size, g = pl->cfg.num_q_heads / pl->cfg.num_kv_heads;
+    if ((D != 64 && D != 128) || (ps != 16 && ps != 32 && ps != 64 && ps != 128) || kRows % g != 0) {
+        *err = "shape outside the tcgen05 kernel's range";
+        return cudaErrorNotSupported;
+    }
+    return D == 128 ? launch_attn_tc_d<128>(pl, k_pool, v_pool, q, out, lse, chunk, st, err)
+                    : launch_attn_tc_d<64>(pl, k_pool, v_pool, q, out, lse, chunk, st, err);
 }
 
 }  // namespace tessera
