@@ -165,11 +165,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     reg_dealloc<80>();
     if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
+        // A tile holds (128 / g) tokens x g heads = q_rows rows; when g does not divide 128 the last
+        // rows of the 128-row MMA tile are padding and are zeroed once (their results are never stored).
+        const int q_rows = (kRows / g) * g;
+        if (q_rows < kRows) {
+            for (int q = 0; q < n_tiles; ++q)
+#pragma unroll
+                for (int hf = 0; hf < G::kHalves; ++hf) {
+                    uint8_t *base = sm + kSmemQ + q * kQTileBytes + hf * kHalfBytes;
+                    for (int o = q_rows * 128 + lane * 16; o < kRows * 128; o += 32 * 16)
+                        *reinterpret_cast<uint4 *>(base + o) = make_uint4(0, 0, 0, 0);
+                }
+            fence_proxy_async_smem();
+            __syncwarp();
+        }
         if (lane == 0) {
             for (int q = 0; q < n_tiles; ++q) {
                 const AttnTile &t = q ? t1 : t0;
                 const uint32_t bar = smem_u32(&bars.q_full[q]);
-                mbar_expect_tx(bar, kQTileBytes);
+                mbar_expect_tx(bar, (uint32_t)(G::kHalves * q_rows * 128));
 #pragma unroll
                 for (int hf = 0; hf < G::kHalves; ++hf)
                     tma_load_3d(smem_u32(sm + kSmemQ + q * kQTileBytes + hf * kHalfBytes), &tmap_q, bar, hf * 64, kvh * g, t.q_begin);
@@ -556,7 +570,7 @@ cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, c
                            float *lse, int chunk, cudaStream_t st, std::string *err) {
     if (pl->n_q == 0 || pl->work.empty()) return cudaSuccess;
     const int D = pl->cfg.head_dim, ps = pl->cfg.page_size, g = pl->cfg.num_q_heads / pl->cfg.num_kv_heads;
-    if ((D != 64 && D != 128) || (ps != 16 && ps != 32 && ps != 64 && ps != 128) || kRows % g != 0) {
+    if ((D != 64 && D != 128) || (ps != 16 && ps != 32 && ps != 64 && ps != 128) || g > 16) {
         *err = "shape outside the tcgen05 kernel's range";
         return cudaErrorNotSupported;
     }

@@ -229,7 +229,7 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
     const int g = Hq / Hkv;
     pl->attn_kernel = 0;
     pl->tile_tokens = kAttnTileRows / g;
-    if (kHaveTensorCoreKernel && (B == 16 || B == 32 || B == 64 || B == 128) && kAttnTileRows % g == 0) pl->attn_kernel = 1;
+    if (kHaveTensorCoreKernel && (B == 16 || B == 32 || B == 64 || B == 128)) pl->attn_kernel = 1;
     pl->tiles.clear();
     for (int r = 0; r < batch; ++r)
         for (int j0 = d->recompute_off[r]; j0 < d->recompute_off[r + 1]; j0 += pl->tile_tokens) {

@@ -430,3 +430,15 @@ def test_residency_decided_by_the_reuse_score_policy():
     recomputed in full inside the same extend pass."""
     w = wl.config(3, requests_override=3, policy="reuse")
     _full_check(w)
+
+
+@pytest.mark.parametrize("hq,hkv,D", [(40, 8, 128), (24, 8, 128), (28, 4, 128), (12, 2, 64)])
+def test_group_sizes_that_do_not_divide_the_tile(hq, hkv, D):
+    """g = 5, 3, 7, 6 query heads per KV head (Qwen-style head counts): a tile holds floor(128 / g)
+    tokens and the remaining MMA rows are zero padding."""
+    shape = wl.ModelShape(hq, hkv, D, 64 if D == 128 else 16, 500000.0)
+    g, _ = _full_check(wl.adversarial(seed=50 + hq, shape=shape))
+    assert g.plan.info.attn_kernel == 1
+    w = wl.build_workload("mid", shape, [[3, wl.unit(700, "a", recompute=range(9)), wl.unit(300, "b", cached=False), 41]],
+                          np.random.default_rng(hq))
+    _full_check(w)
