@@ -123,7 +123,7 @@ typedef struct tessera_plan_info {
     int32_t n_gather_items;     /* thread blocks of the gather kernel                           */
     int32_t n_attn_items;       /* (q tile, kv head) work items of the attention kernel         */
     int32_t attn_kernel;        /* 0 = generic SIMT kernel, 1 = tcgen05 kernel (page_size 16, 32, 64
-                                   or 128 and H_q/H_kv in 1, 2, 4, 8, 16)                                 */
+                                   or 128; any H_q/H_kv up to 16)                                         */
 } tessera_plan_info;
 
 /*
