@@ -154,7 +154,9 @@ TESSERA_API int32_t tessera_plan_get_info(const tessera_plan *plan, tessera_plan
 /*
  * Reads the plan's device status word (synchronises `stream` first).  0 when no kernel of this plan
  * hit a bounded-wait limit since the last call; otherwise TESSERA_DEVICE_TIMEOUT and *detail (host,
- * nullable) receives a code naming the wait.  The word is cleared by the call.
+ * nullable) receives a code naming the wait.  The word is cleared by the call.  While the word is
+ * non-zero the attention kernel's blocks return at once (a stalled launch ends after one round of
+ * timeouts), so after a timeout this call must be made before the plan is used again.
  */
 TESSERA_API int32_t tessera_plan_status(tessera_plan *plan, int32_t *detail, void *stream);
 

@@ -37,6 +37,12 @@ constexpr int kStep = 128;         // keys per step (two pages)
 constexpr int kRows = 128;         // rows per query tile
 constexpr int kRing = 5;           // K/V ring slots
 constexpr int kThreads = 384;        // 8 softmax warps, producer, MMA, 2 idle warps (register donors)
+// setmaxnreg moves registers inside the pool the block got at launch (threads x registers per thread
+// under __launch_bounds__): the raised and lowered counts together must fit in it, or the raise
+// waits forever.
+constexpr int kRegsLaunch = (65536 / kThreads) / 8 * 8;
+constexpr int kRegsSoftmax = 208, kRegsOther = 80;
+static_assert(256 * kRegsSoftmax + 128 * kRegsOther <= kThreads * kRegsLaunch, "register pool of the block exceeded");
 
 // Shared-memory geometry for head_dim D (64 or 128): a tile of 128 rows is stored as D/64 "halves" of
 // [128 rows][128 B] (64 elements per row, 128-byte swizzle).
@@ -113,6 +119,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     __shared__ float s_xchg[2][kRows];              // row maxima exchanged between the two column halves
     __shared__ int s_flag[2][2][4][2];              // [step parity][tile][warp pair][half]
 
+    // A block of a launch in which another block already gave up on a wait does not start, so a
+    // stalled launch ends after one round of timeouts rather than one per block.
+    if (*reinterpret_cast<volatile int *>(status) != 0) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const AttnWork wk = work[blockIdx.x];
     const int n_tiles = wk.tile_b >= 0 ? 2 : 1;
@@ -162,7 +171,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     // Registers move from the producer / MMA warp group to the softmax warps, which hold a whole
     // 128-column row of S plus the packed probabilities.
     if (warp >= 8) {
-    reg_dealloc<80>();
+    reg_dealloc<kRegsOther>();
     if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
         // A tile holds (128 / g) tokens x g heads = q_rows rows; when g does not divide 128 the last
@@ -300,7 +309,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         }
     }
     } else {
-        reg_alloc<208>();
+        reg_alloc<kRegsSoftmax>();
         // ------------------------------------------------------------------ softmax + epilogue
         // All eight warps work on ONE tile at a time and alternate between the tiles: warps 0-3 take
         // columns 0-63 of a row, warps 4-7 columns 64-127 (warp w and w + 4 share TMEM lanes).  The
