@@ -16,6 +16,11 @@
  *                           cached rows placed at request positions with keys
  *                           rotated to the new positions; recomputed rows private
  *                           to the request override cached ones.
+ *   oracle_e4m3_*         - the 8-bit storage form of cached units (1-4-3 float, bias 7, no
+ *                           infinities, maximum 448): decode, and encode with round-to-nearest-
+ *                           even and saturation.  The paper stores conventional 16-bit K/V
+ *                           (Sec. 8); the 8-bit tier is this build's extension and these two
+ *                           functions are its definition.
  *   oracle_attention_rows - the extend pass restricted to the recompute rows
  *                           (Sec. 5.3, Sec. 6.1 "Implementation"): causal softmax
  *                           attention of a query at position p over keys 0..p.
@@ -38,6 +43,57 @@ static double bf16_to_double(uint16_t b) {
     float f;
     memcpy(&f, &u, sizeof f);
     return (double)f;
+}
+
+/* -------------------------------------------------------------------------
+ * 8-bit floating point "e4m3": sign, 4 exponent bits (bias 7), 3 mantissa bits.
+ * Exponent field 0 holds subnormals m * 2^-9; field 15 with mantissa 7 is NaN,
+ * every other pattern is finite (largest 1.75 * 2^8 = 448).  No infinities.
+ * ------------------------------------------------------------------------- */
+double oracle_e4m3_to_double(uint8_t b)
+{
+    int sign = b >> 7, e = (b >> 3) & 15, m = b & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m, -9);
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+/* Nearest representable value, ties to the even mantissa; magnitudes beyond 448 (and
+ * infinities) saturate to +-448; NaN stays NaN.  The input is a float: the decision
+ * is taken on that float exactly (every float is a dyadic rational, so the comparison
+ * with the two neighbouring codes is exact in double arithmetic). */
+uint8_t oracle_f32_to_e4m3(float f)
+{
+    uint8_t sign;
+    double a, lo_v, hi_v;
+    int lo, hi;
+    if (isnan(f)) return 0x7f;
+    sign = signbit(f) ? 0x80 : 0x00;
+    a = fabs((double)f);
+    if (a >= 448.0) return sign | 0x7e;
+    /* codes 0x00..0x7e are increasing in value: bisect for the last code <= a */
+    lo = 0; hi = 0x7e;
+    while (hi - lo > 1) {
+        int mid = (lo + hi) / 2;
+        if (oracle_e4m3_to_double((uint8_t)mid) <= a) lo = mid; else hi = mid;
+    }
+    lo_v = oracle_e4m3_to_double((uint8_t)lo);
+    hi_v = oracle_e4m3_to_double((uint8_t)hi);
+    if (a - lo_v < hi_v - a) return sign | (uint8_t)lo;
+    if (a - lo_v > hi_v - a) return sign | (uint8_t)hi;
+    return sign | (uint8_t)((lo & 1) ? hi : lo);      /* tie: even mantissa */
+}
+
+void oracle_e4m3_decode(const uint8_t *in, double *out, long n)
+{
+    for (long i = 0; i < n; ++i) out[i] = oracle_e4m3_to_double(in[i]);
+}
+
+void oracle_e4m3_encode(const float *in, uint8_t *out, long n)
+{
+    for (long i = 0; i < n; ++i) out[i] = oracle_f32_to_e4m3(in[i]);
 }
 
 /* -------------------------------------------------------------------------
@@ -126,6 +182,32 @@ void oracle_rope_rotate(const double *x, double *out, int D, double delta, doubl
  * k_asm is fp64 and left unrounded.  k_bits / k_exact: rows whose result is a bit
  * copy (recomputed rows and delta == 0) are given as bf16 bits with k_exact = 1.
  * ------------------------------------------------------------------------- */
+static uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40);   /* NaN */
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+/* 8-bit source pools (src_fmt 1; this build's extension, see oracle_e4m3_*): a stored code c
+ * stands for c * scale.  The 16-bit row that reaches the destination is the float product
+ * (float)c * scale rounded to nearest-even bf16 - the precision in which the library takes that
+ * decision - for V and for keys whose shift is 0; rotated keys are computed from the exact
+ * product in fp64 and left unrounded like every other rotated key. */
+int oracle_assemble_ex(int r, const int32_t *seq_len, const int32_t *unit_off,
+                    const int32_t *unit_len, const int32_t *unit_cached_pos,
+                    const int32_t *unit_cached_stride, const int32_t *unit_target_pos,
+                    const int32_t *unit_page_off, const int32_t *unit_pages,
+                    const int32_t *recompute_off, const int32_t *recompute_pos,
+                    int page_size, int H_kv, int D, double theta, const double *inv_freq, int pairing,
+                    const void *k_pool_any, const void *v_pool_any,
+                    const uint16_t *k_new, const uint16_t *v_new,
+                    const int32_t *unit_src_offset /* nullable */, const int32_t *unit_target_stride /* nullable */,
+                    int src_fmt, float k_scale, float v_scale,
+                    double *k_asm, uint16_t *v_asm, uint16_t *k_bits, uint8_t *k_exact, int32_t *delta_out);
+
 int oracle_assemble(int r, const int32_t *seq_len, const int32_t *unit_off,
                     const int32_t *unit_len, const int32_t *unit_cached_pos,
                     const int32_t *unit_cached_stride, const int32_t *unit_target_pos,
@@ -137,6 +219,26 @@ int oracle_assemble(int r, const int32_t *seq_len, const int32_t *unit_off,
                     const int32_t *unit_src_offset /* nullable */, const int32_t *unit_target_stride /* nullable */,
                     double *k_asm, uint16_t *v_asm, uint16_t *k_bits, uint8_t *k_exact, int32_t *delta_out)
 {
+    return oracle_assemble_ex(r, seq_len, unit_off, unit_len, unit_cached_pos, unit_cached_stride, unit_target_pos,
+                              unit_page_off, unit_pages, recompute_off, recompute_pos, page_size, H_kv, D, theta,
+                              inv_freq, pairing, k_pool, v_pool, k_new, v_new, unit_src_offset, unit_target_stride,
+                              0, 1.0f, 1.0f, k_asm, v_asm, k_bits, k_exact, delta_out);
+}
+
+int oracle_assemble_ex(int r, const int32_t *seq_len, const int32_t *unit_off,
+                    const int32_t *unit_len, const int32_t *unit_cached_pos,
+                    const int32_t *unit_cached_stride, const int32_t *unit_target_pos,
+                    const int32_t *unit_page_off, const int32_t *unit_pages,
+                    const int32_t *recompute_off, const int32_t *recompute_pos,
+                    int page_size, int H_kv, int D, double theta, const double *inv_freq, int pairing,
+                    const void *k_pool_any, const void *v_pool_any,
+                    const uint16_t *k_new, const uint16_t *v_new,
+                    const int32_t *unit_src_offset /* nullable */, const int32_t *unit_target_stride /* nullable */,
+                    int src_fmt, float k_scale, float v_scale,
+                    double *k_asm, uint16_t *v_asm, uint16_t *k_bits, uint8_t *k_exact, int32_t *delta_out)
+{
+    const uint16_t *k_pool = (const uint16_t *)k_pool_any, *v_pool = (const uint16_t *)v_pool_any;
+    const uint8_t *k_pool8 = (const uint8_t *)k_pool_any, *v_pool8 = (const uint8_t *)v_pool_any;
     int T = seq_len[r];
     size_t row = (size_t)H_kv * D;
     uint8_t *have = (uint8_t *)calloc((size_t)T + 1, 1);
@@ -151,16 +253,23 @@ int oracle_assemble(int r, const int32_t *seq_len, const int32_t *unit_off,
             int tstride = unit_target_stride ? unit_target_stride[u] : 1;
             int delta = (unit_target_pos[u] + tstride * i) - (unit_cached_pos[u] + unit_cached_stride[u] * i);
             delta_out[p] = delta;
-            memcpy(v_asm + (size_t)p * row, v_pool + slot * row, row * sizeof(uint16_t));
+            if (src_fmt == 0) memcpy(v_asm + (size_t)p * row, v_pool + slot * row, row * sizeof(uint16_t));
+            else
+                for (size_t e = 0; e < row; ++e)
+                    v_asm[(size_t)p * row + e] = f32_to_bf16_rne((float)oracle_e4m3_to_double(v_pool8[slot * row + e]) * v_scale);
             for (int h = 0; h < H_kv; ++h) {
-                const uint16_t *src = k_pool + slot * row + (size_t)h * D;
                 double *dst = k_asm + (size_t)p * row + (size_t)h * D;
-                for (int d = 0; d < D; ++d) tmp[d] = bf16_to_double(src[d]);
+                for (int d = 0; d < D; ++d)
+                    tmp[d] = src_fmt == 0 ? bf16_to_double(k_pool[slot * row + (size_t)h * D + d])
+                                          : oracle_e4m3_to_double(k_pool8[slot * row + (size_t)h * D + d]) * (double)k_scale;
                 oracle_rope_rotate(tmp, dst, D, (double)delta, theta, inv_freq, pairing);
             }
             if (delta == 0) {
                 k_exact[p] = 1;
-                memcpy(k_bits + (size_t)p * row, k_pool + slot * row, row * sizeof(uint16_t));
+                if (src_fmt == 0) memcpy(k_bits + (size_t)p * row, k_pool + slot * row, row * sizeof(uint16_t));
+                else
+                    for (size_t e = 0; e < row; ++e)
+                        k_bits[(size_t)p * row + e] = f32_to_bf16_rne((float)oracle_e4m3_to_double(k_pool8[slot * row + e]) * k_scale);
             }
             have[p] = 1;
         }

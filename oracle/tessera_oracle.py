@@ -35,6 +35,9 @@ def lib():
         _lib = ctypes.CDLL(build())
         _lib.oracle_placement.restype = ctypes.c_int
         _lib.oracle_assemble.restype = ctypes.c_int
+        _lib.oracle_assemble_ex.restype = ctypes.c_int
+        _lib.oracle_e4m3_decode.restype = None
+        _lib.oracle_e4m3_encode.restype = None
         _lib.oracle_num_threads.restype = ctypes.c_int
         _lib.oracle_rope_rotate.restype = None
         _lib.oracle_attention_rows.restype = None
@@ -110,14 +113,33 @@ class Assembled:
         self.delta = np.zeros(T, np.int32)
 
 
+def e4m3_decode(codes: np.ndarray) -> np.ndarray:
+    """uint8 e4m3 codes -> float64 values (NaN for the NaN code)."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    out = np.empty(codes.shape, np.float64)
+    lib().oracle_e4m3_decode(_p(codes), _p(out), ctypes.c_long(codes.size))
+    return out
+
+
+def e4m3_encode(values: np.ndarray) -> np.ndarray:
+    """float32 values -> uint8 e4m3 codes: nearest, ties to even, saturating at +-448."""
+    values = np.ascontiguousarray(values, dtype=np.float32)
+    out = np.empty(values.shape, np.uint8)
+    lib().oracle_e4m3_encode(_p(values), _p(out), ctypes.c_long(values.size))
+    return out
+
+
 def assemble(w, r: int, k_pool_bits, v_pool_bits, k_new_bits, v_new_bits,
-             inv_freq: Optional[np.ndarray] = None) -> Assembled:
+             inv_freq: Optional[np.ndarray] = None, src_fmt: int = 0, k_scale: float = 1.0,
+             v_scale: float = 1.0) -> Assembled:
+    """src_fmt 0: 16-bit source pools given as bf16 bits; 1: 8-bit (e4m3 codes, uint8) source pools,
+    a code standing for code * scale."""
     sh = w.shape
     T = int(w.seq_len[r])
     a = Assembled(T, sh.num_kv_heads, sh.head_dim)
     if inv_freq is not None:
         inv_freq = np.ascontiguousarray(inv_freq, dtype=np.float64)
-    st = lib().oracle_assemble(
+    st = lib().oracle_assemble_ex(
         ctypes.c_int(r), _p(_i32(w.seq_len)), _p(_i32(w.unit_off)), _p(_i32(w.unit_len)),
         _p(_i32(w.unit_cached_pos)), _p(_i32(w.unit_cached_stride)), _p(_i32(w.unit_target_pos)),
         _p(_i32(w.unit_page_off)), _p(_i32(w.unit_pages)), _p(_i32(w.recompute_off)),
@@ -126,6 +148,7 @@ def assemble(w, r: int, k_pool_bits, v_pool_bits, k_new_bits, v_new_bits,
         ctypes.c_int(sh.rope_pairing),
         _p(k_pool_bits), _p(v_pool_bits), _p(k_new_bits), _p(v_new_bits),
         _p(_opt(w, "unit_src_offset")), _p(_opt(w, "unit_target_stride")),
+        ctypes.c_int(src_fmt), ctypes.c_float(k_scale), ctypes.c_float(v_scale),
         _p(a.k), _p(a.v_bits), _p(a.k_bits), _p(a.k_exact), _p(a.delta))
     if st != 0:
         raise ValueError("oracle_assemble: request %d has positions nobody supplies" % r)

@@ -322,3 +322,68 @@ def test_kv_byte_model_closed_form():
     w = wl.config(2)
     assert w.total_tokens == 5312 and w.n_q == 352 and w.cached_tokens == 5120
     assert wl.gather_bytes(w) == 5120 * 8192
+
+
+# ---------------------------------------------------------------- 8-bit (e4m3) storage form
+def test_e4m3_decode_all_codes_against_library_and_closed_forms():
+    codes = np.arange(256, dtype=np.uint8)
+    v = orc.e4m3_decode(codes)
+    lib = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).double().numpy()
+    assert np.array_equal(np.isnan(v), np.isnan(lib)) and np.isnan(v).sum() == 2
+    assert np.array_equal(v[~np.isnan(v)], lib[~np.isnan(lib)])
+    assert v[0x38] == 1.0 and v[0x7e] == 448.0 and v[0x01] == 2.0 ** -9 and v[0x08] == 2.0 ** -6
+    assert v[0xb8] == -1.0 and v[0x80] == 0.0 and np.signbit(v[0x80])
+    assert np.all(np.diff(v[:0x7f]) > 0)                      # codes 0x00..0x7e ascend
+
+
+def test_e4m3_encode_nearest_even_saturating():
+    table = orc.e4m3_decode(np.arange(0x7f, dtype=np.uint8))
+    # round trip of every finite code, both signs
+    assert np.array_equal(orc.e4m3_encode(table.astype(np.float32)), np.arange(0x7f, dtype=np.uint8))
+    assert np.array_equal(orc.e4m3_encode((-table).astype(np.float32)), np.arange(0x7f, dtype=np.uint8) | 0x80)
+    # exact midpoints go to the even code; a hair to either side goes to the nearer one
+    mid = ((table[:-1] + table[1:]) / 2).astype(np.float32)
+    assert np.array_equal(mid.astype(np.float64), (table[:-1] + table[1:]) / 2)     # midpoints are floats
+    lo = np.arange(0x7e, dtype=np.uint8)
+    assert np.array_equal(orc.e4m3_encode(mid), np.where(lo % 2 == 0, lo, lo + 1))
+    assert np.array_equal(orc.e4m3_encode(np.nextafter(mid, np.float32(0))), lo)
+    assert np.array_equal(orc.e4m3_encode(np.nextafter(mid, np.float32(1e9))), lo + 1)
+    # saturation and NaN
+    big = np.array([448.0, 449.0, 464.0, 1e9, np.inf, -1e9, -np.inf, np.nan], np.float32)
+    assert orc.e4m3_encode(big).tolist() == [0x7e, 0x7e, 0x7e, 0x7e, 0x7e, 0xfe, 0xfe, 0x7f]
+    # library conversion (which does not saturate) on values inside the range
+    rng = np.random.default_rng(0)
+    x = (rng.standard_normal(100000) * np.exp(rng.uniform(-12, 5, 100000))).astype(np.float32)
+    x = x[np.abs(x) < 448]
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(orc.e4m3_encode(x), want)
+
+
+def test_assemble_from_8bit_pool_reduces_to_the_16bit_path():
+    """Every e4m3 value (and its product with a power of two) is a bf16 value, so an 8-bit source pool
+    with a power-of-two scale must assemble exactly like the 16-bit pool holding the same numbers."""
+    w = wl.adversarial()
+    t = wl.make_tensors(w, seed=5)
+    rng = np.random.default_rng(2)
+    knb, vnb = orc.bits(t.k_new), orc.bits(t.v_new)
+    shape = tuple(t.k_pool.shape)
+    k8 = rng.integers(0, 256, size=shape, dtype=np.uint8)
+    v8 = rng.integers(0, 256, size=shape, dtype=np.uint8)
+    k8[(k8 & 0x7f) == 0x7f] = 0x38                            # no NaN codes
+    v8[(v8 & 0x7f) == 0x7f] = 0x38
+    for scale in (1.0, 0.25):
+        kb = orc.bits(torch.from_numpy(orc.e4m3_decode(k8) * scale).to(torch.bfloat16))
+        vb = orc.bits(torch.from_numpy(orc.e4m3_decode(v8) * scale).to(torch.bfloat16))
+        assert np.array_equal(orc.bf16_bits_to_f64(kb), orc.e4m3_decode(k8) * scale)     # exact in bf16
+        for r in range(w.batch):
+            a16 = orc.assemble(w, r, kb, vb, knb, vnb)
+            a8 = orc.assemble(w, r, k8, v8, knb, vnb, src_fmt=1, k_scale=scale, v_scale=scale)
+            assert np.array_equal(a16.v_bits, a8.v_bits) and np.array_equal(a16.k, a8.k)
+            assert np.array_equal(a16.k_exact, a8.k_exact) and np.array_equal(a16.k_bits, a8.k_bits)
+    # a scale that is not a power of two: the 16-bit row is the float product rounded once more to bf16
+    a8 = orc.assemble(w, 0, k8, v8, knb, vnb, src_fmt=1, k_scale=0.3, v_scale=0.7)
+    st, _, _, src_slot, fresh = orc.placement(w)
+    row = w.shape.num_kv_heads * w.shape.head_dim
+    p = next(p for p in range(int(w.seq_len[0])) if fresh[p] < 0)
+    want = (orc.e4m3_decode(v8.reshape(-1, row)[src_slot[p]]).astype(np.float32) * np.float32(0.7))
+    assert np.array_equal(a8.v_bits[p].ravel(), orc.bits(torch.from_numpy(want).to(torch.bfloat16)))
