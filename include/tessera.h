@@ -185,6 +185,38 @@ TESSERA_API int32_t tessera_kv_compose_from(const tessera_plan *plan, const void
                                             void *k_pool, void *v_pool, uint32_t flags, void *stream);
 
 /*
+ * 8-bit storage tier for cached units.  The paper's system stores conventional 16-bit K/V (Sec. 8,
+ * "Algorithm and Model Compatibility") and has no counterpart of these two calls; they halve the
+ * bytes a cache hit moves (Sec. 2.4: transfer volume is what a hit costs).  A stored byte is an
+ * e4m3 code c (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities, largest finite
+ * value 448, 0x7f / 0xff = NaN) and stands for c * scale, one positive finite scale per pool and
+ * tensor (k_scale, v_scale).  Both calls need a plan created with desc.num_source_pages > 0 and use
+ * its copy list and shift table exactly as tessera_kv_compose_from does.
+ *
+ * tessera_kv_compose_from_fp8 - expand: k_src8 / v_src8 [num_source_pages][page_size][H_kv][D] bytes
+ *   (device-addressable, 16-byte aligned, never written) -> the request's destination pages in the
+ *   16-bit pools k_pool / v_pool.  V and un-shifted K rows: bf16_rne(fp32(c) * scale) (the fp32
+ *   product is rounded once, then once more to bf16; exact when scale is a power of two).  With
+ *   TESSERA_FUSE_ROPE shifted K rows are rotated in fp32 from those fp32 products and rounded once
+ *   to bf16; without it every K row is treated as un-shifted and tessera_rope_shift must follow.
+ *
+ * tessera_kv_retain_fp8 - retain: the reverse direction.  k_src / v_src are 16-bit pools
+ *   [num_source_pages] (e.g. a finished request's pages), k_dst8 / v_dst8 8-bit pools of
+ *   num_pool_pages pages whose free pages the plan consumed.  Every element is (rotated by the
+ *   plan's shift when TESSERA_FUSE_ROPE is given - a retention plan shifts keys back to their
+ *   position-free form -) multiplied in fp32 by the fp32 reciprocal 1.0f / scale and rounded to the
+ *   nearest e4m3 value, ties to even, magnitudes above 448 saturating to +-448, NaN to 0x7f.
+ *
+ * Errors: as tessera_kv_compose_from; TESSERA_INVALID_ARG also for a scale that is not positive and
+ * finite.  Nothing is allocated; one kernel is launched on `stream`.
+ */
+TESSERA_API int32_t tessera_kv_compose_from_fp8(const tessera_plan *plan, const void *k_src8, const void *v_src8,
+                                                float k_scale, float v_scale, void *k_pool, void *v_pool,
+                                                uint32_t flags, void *stream);
+TESSERA_API int32_t tessera_kv_retain_fp8(const tessera_plan *plan, const void *k_src, const void *v_src, void *k_dst8,
+                                          void *v_dst8, float k_scale, float v_scale, uint32_t flags, void *stream);
+
+/*
  * "Applying RoPE to the keys at their new positions" (Sec. 5.3; the fused placement kernel of
  * Sec. 6.1) as a call of its own: rotates, in place, the destination-page K rows of every cached
  * unit by (new position - cached position).  NOT idempotent: call exactly once after a compose

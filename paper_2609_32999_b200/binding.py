@@ -53,7 +53,7 @@ class PlanInfo(ctypes.Structure):
 
 
 EXPORTS = ["tessera_plan_create", "tessera_plan_destroy", "tessera_plan_block_table", "tessera_plan_get_info",
-           "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_rope_shift", "tessera_rope_fresh", "tessera_partial_prefill_attn",
+           "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_kv_compose_from_fp8", "tessera_kv_retain_fp8", "tessera_rope_shift", "tessera_rope_fresh", "tessera_partial_prefill_attn",
            "tessera_composed_prefill_host", "tessera_rope_shift_static", "tessera_selftest_bounded_wait", "tessera_last_error",
            "tessera_launch_count"]
 
@@ -66,6 +66,8 @@ _lib.tessera_plan_get_info.argtypes = [_vp, ctypes.POINTER(PlanInfo)]
 _lib.tessera_plan_status.argtypes = [_vp, _I32P, _vp]
 _lib.tessera_kv_compose.argtypes = [_vp, _vp, _vp, ctypes.c_uint32, _vp]
 _lib.tessera_kv_compose_from.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_uint32, _vp]
+_lib.tessera_kv_compose_from_fp8.argtypes = [_vp, _vp, _vp, ctypes.c_float, ctypes.c_float, _vp, _vp, ctypes.c_uint32, _vp]
+_lib.tessera_kv_retain_fp8.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, _vp]
 _lib.tessera_rope_shift.argtypes = [_vp, _vp, _vp]
 _lib.tessera_rope_fresh.argtypes = [_vp, _vp, _vp, _vp]
 _lib.tessera_partial_prefill_attn.argtypes = [_vp] * 9
@@ -178,6 +180,18 @@ class Plan:
         """Sources in a separate pool (pinned host tensors or device tensors), destinations in the pools."""
         _check(_lib.tessera_kv_compose_from(self._h, _dev(k_src), _dev(v_src), _dev(k_pool), _dev(v_pool),
                                             FUSE_ROPE if fuse_rope else 0, _stream(stream)))
+
+    def kv_compose_from_fp8(self, k_src8, v_src8, k_scale: float, v_scale: float, k_pool, v_pool,
+                            fuse_rope: bool = True, stream=None) -> None:
+        """Sources are e4m3 codes (uint8 or float8_e4m3fn tensors) standing for code * scale."""
+        _check(_lib.tessera_kv_compose_from_fp8(self._h, _dev(k_src8), _dev(v_src8), k_scale, v_scale, _dev(k_pool),
+                                                _dev(v_pool), FUSE_ROPE if fuse_rope else 0, _stream(stream)))
+
+    def kv_retain_fp8(self, k_src, v_src, k_dst8, v_dst8, k_scale: float, v_scale: float, fuse_rope: bool = True,
+                      stream=None) -> None:
+        """16-bit source pools -> e4m3 destination pools (the plan's destination pages index the 8-bit pools)."""
+        _check(_lib.tessera_kv_retain_fp8(self._h, _dev(k_src), _dev(v_src), _dev(k_dst8), _dev(v_dst8), k_scale, v_scale,
+                                          FUSE_ROPE if fuse_rope else 0, _stream(stream)))
 
     def rope_shift(self, k_pool, stream=None) -> None:
         _check(_lib.tessera_rope_shift(self._h, _dev(k_pool), _stream(stream)))

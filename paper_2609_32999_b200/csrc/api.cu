@@ -4,6 +4,7 @@
 #include <new>
 #include <string>
 
+#include <cmath>
 #include <cuda_runtime.h>
 
 #include "launch.h"
@@ -270,6 +271,38 @@ int32_t tessera_kv_compose_from(const tessera_plan *pl, const void *k_src, const
         return set_error(TESSERA_INVALID_ARG, "k_src / v_src / k_pool / v_pool must be non-null and 16-byte aligned");
     TS_CUDA(launch_gather(pl, k_src, v_src, k_pool, v_pool, (flags & TESSERA_FUSE_ROPE) ? GatherMode::kCopyRotate : GatherMode::kCopy,
                           static_cast<cudaStream_t>(stream)));
+    return TESSERA_OK;
+}
+
+namespace {
+int32_t check_fp8_call(const tessera_plan *pl, const void *a, const void *b, const void *c, const void *d, uint32_t flags,
+                       float k_scale, float v_scale) {
+    if (int32_t rc = check_device_plan(pl)) return rc;
+    if (flags & ~uint32_t(TESSERA_FUSE_ROPE)) return set_error(TESSERA_INVALID_ARG, "unknown compose flag");
+    if (pl->num_source_pages <= 0)
+        return set_error(TESSERA_INVALID_ARG, "the plan was created without a separate source pool (desc.num_source_pages)");
+    if (!a || !b || !c || !d || misaligned(a) || misaligned(b) || misaligned(c) || misaligned(d))
+        return set_error(TESSERA_INVALID_ARG, "source and destination pools must be non-null and 16-byte aligned");
+    if (!(k_scale > 0.f) || !(v_scale > 0.f) || std::isinf(k_scale) || std::isinf(v_scale))
+        return set_error(TESSERA_INVALID_ARG, "k_scale / v_scale must be positive and finite");
+    return TESSERA_OK;
+}
+}  // namespace
+
+int32_t tessera_kv_compose_from_fp8(const tessera_plan *pl, const void *k_src8, const void *v_src8, float k_scale,
+                                    float v_scale, void *k_pool, void *v_pool, uint32_t flags, void *stream) {
+    if (int32_t rc = check_fp8_call(pl, k_src8, v_src8, k_pool, v_pool, flags, k_scale, v_scale)) return rc;
+    TS_CUDA(launch_kv_fp8(pl, k_src8, v_src8, k_pool, v_pool, false, (flags & TESSERA_FUSE_ROPE) != 0, k_scale, v_scale,
+                          static_cast<cudaStream_t>(stream)));
+    return TESSERA_OK;
+}
+
+int32_t tessera_kv_retain_fp8(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst8, void *v_dst8,
+                              float k_scale, float v_scale, uint32_t flags, void *stream) {
+    if (int32_t rc = check_fp8_call(pl, k_src, v_src, k_dst8, v_dst8, flags, k_scale, v_scale)) return rc;
+    // the reciprocal is taken once, in fp32: every element is multiplied by it (one rounding) and then rounded to e4m3
+    TS_CUDA(launch_kv_fp8(pl, k_src, v_src, k_dst8, v_dst8, true, (flags & TESSERA_FUSE_ROPE) != 0, 1.0f / k_scale,
+                          1.0f / v_scale, static_cast<cudaStream_t>(stream)));
     return TESSERA_OK;
 }
 

@@ -1,0 +1,197 @@
+// Cached units stored as 8-bit floats (e4m3: 4 exponent bits, 3 mantissa bits, no infinities, largest
+// value 448; a stored code c stands for c * scale, one scale per pool).  The paper's system keeps
+// conventional 16-bit K/V (Sec. 8); this tier halves the bytes a cache hit moves (Sec. 2.4) and is
+// this library's extension.  Two directions, both driven by the plan's copy list and shift table:
+//   expand : 8-bit source pool -> the request's 16-bit pages (keys rotated on the way, Sec. 5.3)
+//   retain : 16-bit pages -> 8-bit storage pages (keys rotated by the plan's shifts - normally back
+//            to the position-free form - then scaled and rounded to nearest-even, saturating)
+// A task is the same pair-chunk as in the 16-bit gather: 8 elements of a head and their partners
+// D/2 elements later - 8-byte accesses on the 8-bit side, 16-byte accesses on the 16-bit side.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
+#include <cuda_runtime.h>
+
+#include "launch.h"
+#include "plan.h"
+
+namespace tessera {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ void unpack_bf16x8(const uint4 &v, float (&f)[8]) {
+    const uint32_t *w = reinterpret_cast<const uint32_t *>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[2 * i] = __uint_as_float(w[i] << 16);
+        f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+__device__ __forceinline__ uint4 pack_bf16x8(const float (&f)[8]) {
+    uint4 v;
+    uint32_t *w = reinterpret_cast<uint32_t *>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t *>(&p);
+    }
+    return v;
+}
+// 8 codes -> 8 floats (exact) times mul (one fp32 rounding).
+__device__ __forceinline__ void unpack_e4m3x8(const uint2 &v, float mul, float (&f)[8]) {
+    const uint32_t w[2] = {v.x, v.y};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_fp8x2_storage_t two = (__nv_fp8x2_storage_t)((w[i >> 1] >> (16 * (i & 1))) & 0xffffu);
+        const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2(two, __NV_E4M3);
+        const float2 x = __half22float2(*reinterpret_cast<const __half2 *>(&h));
+        f[2 * i] = __fmul_rn(x.x, mul);
+        f[2 * i + 1] = __fmul_rn(x.y, mul);
+    }
+}
+// 8 floats times mul (one fp32 rounding) -> 8 codes, nearest-even, saturating at +-448.
+__device__ __forceinline__ uint2 pack_e4m3x8(const float (&f)[8], float mul) {
+    uint32_t w[2] = {0u, 0u};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 x = make_float2(__fmul_rn(f[2 * i], mul), __fmul_rn(f[2 * i + 1], mul));
+        const uint32_t two = (uint32_t)__nv_cvt_float2_to_fp8x2(x, __NV_SATFINITE, __NV_E4M3);
+        w[i >> 1] |= two << (16 * (i & 1));
+    }
+    return make_uint2(w[0], w[1]);
+}
+
+// x' = x cos - y sin, y' = y cos + x sin in fp32, the arithmetic of the 16-bit gather.
+template <bool INTERLEAVED>
+__device__ __forceinline__ void rotate_f(float (&lo)[8], float (&hi)[8], const float2 *cs) {
+    if (INTERLEAVED) {
+        // lo holds pairs (0,1) (2,3) .. with cs[0..3]; hi the chunk D/2 elements later with cs[4..7]
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float x = lo[2 * i], y = lo[2 * i + 1], u = hi[2 * i], v = hi[2 * i + 1];
+            lo[2 * i] = fmaf(-y, cs[i].y, x * cs[i].x);
+            lo[2 * i + 1] = fmaf(x, cs[i].y, y * cs[i].x);
+            hi[2 * i] = fmaf(-v, cs[4 + i].y, u * cs[4 + i].x);
+            hi[2 * i + 1] = fmaf(u, cs[4 + i].y, v * cs[4 + i].x);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float x = lo[i], y = hi[i];
+            lo[i] = fmaf(-y, cs[i].y, x * cs[i].x);
+            hi[i] = fmaf(x, cs[i].y, y * cs[i].x);
+        }
+    }
+}
+template <int D, bool INTERLEAVED>
+__device__ __forceinline__ int cs_index(int c, int i) {
+    return INTERLEAVED ? (i < 4 ? 4 * c + i : 4 * c + D / 4 + (i - 4)) : c * 8 + i;
+}
+
+// One thread block per GatherItem.  TO_8BIT false: sources are e4m3 (mul = scale), destinations bf16;
+// TO_8BIT true: sources are bf16, destinations e4m3 (mul = 1 / scale, applied after the rotation).
+template <int D, bool TO_8BIT, bool ROTATE, bool INTERLEAVED>
+__global__ void __launch_bounds__(kThreads)
+kv_fp8_kernel(const void *__restrict__ k_src, const void *__restrict__ v_src, void *__restrict__ k_dst,
+              void *__restrict__ v_dst, const int32_t *__restrict__ g_src, const int32_t *__restrict__ g_dst,
+              const GatherItem *__restrict__ items, const float2 *__restrict__ rope, int H_kv, float k_mul, float v_mul) {
+    constexpr int CPH = D / 16;          // pair-chunks per head
+    constexpr int HALF = D / 16;         // distance (in 8-element chunks) between pair partners
+    __shared__ float2 s_rope[kGatherItemTokens * (D / 2)];
+    __shared__ int32_t s_src[kGatherItemTokens], s_dst[kGatherItemTokens];
+
+    const GatherItem it = items[blockIdx.x];
+    const int tid = threadIdx.x;
+    const int n_rows = ROTATE ? (it.row_step ? it.count : 1) : 0;
+    const int first_row = it.row_step < 0 ? it.row0 - (it.count - 1) : it.row0;
+    for (int i = tid; i < n_rows * (D / 2); i += kThreads) s_rope[i] = rope[(size_t)first_row * (D / 2) + i];
+    if (tid < it.count) {
+        s_dst[tid] = g_dst[it.begin + tid];
+        s_src[tid] = g_src[it.begin + tid];
+    }
+    __syncthreads();
+
+    const int tasks_per_row = H_kv * CPH;
+    const int row_chunks = H_kv * (D / 8);
+    const int n_tasks = it.count * tasks_per_row;
+    const int c = tid % CPH;
+    for (int t = tid; t < n_tasks; t += kThreads) {
+        const int tok = t / tasks_per_row;
+        const int w = t - tok * tasks_per_row;
+        const int chunk = (w / CPH) * (D / 8) + c;
+        const size_t so = (size_t)s_src[tok] * row_chunks + chunk, dso = (size_t)s_dst[tok] * row_chunks + chunk;
+        float klo[8], khi[8], vlo[8], vhi[8];
+        if (TO_8BIT) {
+            const uint4 *ks = static_cast<const uint4 *>(k_src), *vs = static_cast<const uint4 *>(v_src);
+            unpack_bf16x8(ks[so], klo);
+            unpack_bf16x8(ks[so + HALF], khi);
+            unpack_bf16x8(vs[so], vlo);
+            unpack_bf16x8(vs[so + HALF], vhi);
+        } else {
+            const uint2 *ks = static_cast<const uint2 *>(k_src), *vs = static_cast<const uint2 *>(v_src);
+            unpack_e4m3x8(ks[so], k_mul, klo);
+            unpack_e4m3x8(ks[so + HALF], k_mul, khi);
+            unpack_e4m3x8(vs[so], v_mul, vlo);
+            unpack_e4m3x8(vs[so + HALF], v_mul, vhi);
+        }
+        if (ROTATE) {
+            const int sr = it.row_step == 0 ? 0 : (it.row_step < 0 ? it.count - 1 - tok : tok);
+            const float2 *row = s_rope + (size_t)sr * (D / 2);
+            float2 cr[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) cr[i] = row[cs_index<D, INTERLEAVED>(c, i)];
+            rotate_f<INTERLEAVED>(klo, khi, cr);
+        }
+        if (TO_8BIT) {
+            uint2 *kd = static_cast<uint2 *>(k_dst), *vd = static_cast<uint2 *>(v_dst);
+            kd[dso] = pack_e4m3x8(klo, k_mul);
+            kd[dso + HALF] = pack_e4m3x8(khi, k_mul);
+            vd[dso] = pack_e4m3x8(vlo, v_mul);
+            vd[dso + HALF] = pack_e4m3x8(vhi, v_mul);
+        } else {
+            uint4 *kd = static_cast<uint4 *>(k_dst), *vd = static_cast<uint4 *>(v_dst);
+            kd[dso] = pack_bf16x8(klo);
+            kd[dso + HALF] = pack_bf16x8(khi);
+            vd[dso] = pack_bf16x8(vlo);
+            vd[dso + HALF] = pack_bf16x8(vhi);
+        }
+    }
+}
+
+template <int D, bool TO_8BIT, bool IL>
+cudaError_t launch_d(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst, bool rotate,
+                     float k_mul, float v_mul, cudaStream_t st) {
+    const int n = (int)pl->items.size();
+    if (n == 0) return cudaSuccess;
+    const DeviceTables &d = pl->dev;
+    const int H = pl->cfg.num_kv_heads;
+    if (rotate)
+        kv_fp8_kernel<D, TO_8BIT, true, IL><<<n, kThreads, 0, st>>>(k_src, v_src, k_dst, v_dst, d.g_src, d.g_dst, d.items, d.rope, H, k_mul, v_mul);
+    else
+        kv_fp8_kernel<D, TO_8BIT, false, IL><<<n, kThreads, 0, st>>>(k_src, v_src, k_dst, v_dst, d.g_src, d.g_dst, d.items, d.rope, H, k_mul, v_mul);
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <bool TO_8BIT>
+cudaError_t launch_dir(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst, bool rotate,
+                       float k_mul, float v_mul, cudaStream_t st) {
+    const bool il = pl->cfg.rope_pairing == 1;
+    if (pl->cfg.head_dim == 128)
+        return il ? launch_d<128, TO_8BIT, true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st)
+                  : launch_d<128, TO_8BIT, false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st);
+    return il ? launch_d<64, TO_8BIT, true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st)
+              : launch_d<64, TO_8BIT, false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st);
+}
+
+}  // namespace
+
+cudaError_t launch_kv_fp8(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst,
+                          bool to_8bit, bool rotate, float k_mul, float v_mul, cudaStream_t st) {
+    return to_8bit ? launch_dir<true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st)
+                   : launch_dir<false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st);
+}
+
+}  // namespace tessera

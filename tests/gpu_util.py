@@ -73,7 +73,8 @@ def check_placement(g):
 
 def check_assembled(g, requests=None, scattered=True):
     """Destination pages vs the oracle's assembled KV.  Returns (assembled list, max, mean) where
-    max / mean are over all rotated key elements."""
+    max / mean are over all rotated key elements.  g.src_fmt = 1 (with g.k_scale / g.v_scale): the
+    sources in g.k_before / g.v_before are e4m3 codes of an 8-bit pool."""
     w = g.w
     sh = w.shape
     row = sh.num_kv_heads * sh.head_dim
@@ -82,7 +83,8 @@ def check_assembled(g, requests=None, scattered=True):
     asm = {}
     errs = []
     for r in (range(w.batch) if requests is None else requests):
-        a = orc.assemble(w, r, g.k_before, g.v_before, g.kn_bits, g.vn_bits)
+        a = orc.assemble(w, r, g.k_before, g.v_before, g.kn_bits, g.vn_bits, src_fmt=getattr(g, "src_fmt", 0),
+                         k_scale=getattr(g, "k_scale", 1.0), v_scale=getattr(g, "v_scale", 1.0))
         asm[r] = a
         T = int(w.seq_len[r])
         if T == 0:
