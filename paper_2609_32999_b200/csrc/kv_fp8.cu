@@ -12,6 +12,8 @@
 #include <cuda_fp8.h>
 #include <cuda_runtime.h>
 
+#include <type_traits>
+
 #include "launch.h"
 #include "plan.h"
 
@@ -117,45 +119,65 @@ kv_fp8_kernel(const void *__restrict__ k_src, const void *__restrict__ v_src, vo
     const int row_chunks = H_kv * (D / 8);
     const int n_tasks = it.count * tasks_per_row;
     const int c = tid % CPH;
-    for (int t = tid; t < n_tasks; t += kThreads) {
-        const int tok = t / tasks_per_row;
-        const int w = t - tok * tasks_per_row;
-        const int chunk = (w / CPH) * (D / 8) + c;
-        const size_t so = (size_t)s_src[tok] * row_chunks + chunk, dso = (size_t)s_dst[tok] * row_chunks + chunk;
-        float klo[8], khi[8], vlo[8], vhi[8];
-        if (TO_8BIT) {
-            const uint4 *ks = static_cast<const uint4 *>(k_src), *vs = static_cast<const uint4 *>(v_src);
-            unpack_bf16x8(ks[so], klo);
-            unpack_bf16x8(ks[so + HALF], khi);
-            unpack_bf16x8(vs[so], vlo);
-            unpack_bf16x8(vs[so + HALF], vhi);
-        } else {
-            const uint2 *ks = static_cast<const uint2 *>(k_src), *vs = static_cast<const uint2 *>(v_src);
-            unpack_e4m3x8(ks[so], k_mul, klo);
-            unpack_e4m3x8(ks[so + HALF], k_mul, khi);
-            unpack_e4m3x8(vs[so], v_mul, vlo);
-            unpack_e4m3x8(vs[so + HALF], v_mul, vhi);
-        }
-        if (ROTATE) {
-            const int sr = it.row_step == 0 ? 0 : (it.row_step < 0 ? it.count - 1 - tok : tok);
-            const float2 *row = s_rope + (size_t)sr * (D / 2);
-            float2 cr[8];
+    using Raw = typename std::conditional<TO_8BIT, uint4, uint2>::type;   // one 8-element chunk of the source
+    const Raw *ks = static_cast<const Raw *>(k_src), *vs = static_cast<const Raw *>(v_src);
+    constexpr int U = 2;                 // tasks in flight per thread: all loads of both are issued first
+    for (int t0 = tid; t0 < n_tasks; t0 += U * kThreads) {
+        Raw rk[U][2], rv[U][2];
+        size_t dso[U];
+        int tok[U];
+        bool ok[U];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) cr[i] = row[cs_index<D, INTERLEAVED>(c, i)];
-            rotate_f<INTERLEAVED>(klo, khi, cr);
+        for (int u = 0; u < U; ++u) {
+            const int t = t0 + u * kThreads;
+            ok[u] = t < n_tasks;
+            if (!ok[u]) continue;
+            tok[u] = t / tasks_per_row;
+            const int w = t - tok[u] * tasks_per_row;
+            const int chunk = (w / CPH) * (D / 8) + c;
+            const size_t so = (size_t)s_src[tok[u]] * row_chunks + chunk;
+            dso[u] = (size_t)s_dst[tok[u]] * row_chunks + chunk;
+            rk[u][0] = __ldg(ks + so);
+            rk[u][1] = __ldg(ks + so + HALF);
+            rv[u][0] = __ldg(vs + so);
+            rv[u][1] = __ldg(vs + so + HALF);
         }
-        if (TO_8BIT) {
-            uint2 *kd = static_cast<uint2 *>(k_dst), *vd = static_cast<uint2 *>(v_dst);
-            kd[dso] = pack_e4m3x8(klo, k_mul);
-            kd[dso + HALF] = pack_e4m3x8(khi, k_mul);
-            vd[dso] = pack_e4m3x8(vlo, v_mul);
-            vd[dso + HALF] = pack_e4m3x8(vhi, v_mul);
-        } else {
-            uint4 *kd = static_cast<uint4 *>(k_dst), *vd = static_cast<uint4 *>(v_dst);
-            kd[dso] = pack_bf16x8(klo);
-            kd[dso + HALF] = pack_bf16x8(khi);
-            vd[dso] = pack_bf16x8(vlo);
-            vd[dso + HALF] = pack_bf16x8(vhi);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (!ok[u]) continue;
+            float klo[8], khi[8], vlo[8], vhi[8];
+            if constexpr (TO_8BIT) {
+                unpack_bf16x8(rk[u][0], klo);
+                unpack_bf16x8(rk[u][1], khi);
+                unpack_bf16x8(rv[u][0], vlo);
+                unpack_bf16x8(rv[u][1], vhi);
+            } else {
+                unpack_e4m3x8(rk[u][0], k_mul, klo);
+                unpack_e4m3x8(rk[u][1], k_mul, khi);
+                unpack_e4m3x8(rv[u][0], v_mul, vlo);
+                unpack_e4m3x8(rv[u][1], v_mul, vhi);
+            }
+            if (ROTATE) {
+                const int sr = it.row_step == 0 ? 0 : (it.row_step < 0 ? it.count - 1 - tok[u] : tok[u]);
+                const float2 *row = s_rope + (size_t)sr * (D / 2);
+                float2 cr[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) cr[i] = row[cs_index<D, INTERLEAVED>(c, i)];
+                rotate_f<INTERLEAVED>(klo, khi, cr);
+            }
+            if constexpr (TO_8BIT) {
+                uint2 *kd = static_cast<uint2 *>(k_dst), *vd = static_cast<uint2 *>(v_dst);
+                kd[dso[u]] = pack_e4m3x8(klo, k_mul);
+                kd[dso[u] + HALF] = pack_e4m3x8(khi, k_mul);
+                vd[dso[u]] = pack_e4m3x8(vlo, v_mul);
+                vd[dso[u] + HALF] = pack_e4m3x8(vhi, v_mul);
+            } else {
+                uint4 *kd = static_cast<uint4 *>(k_dst), *vd = static_cast<uint4 *>(v_dst);
+                kd[dso[u]] = pack_bf16x8(klo);
+                kd[dso[u] + HALF] = pack_bf16x8(khi);
+                vd[dso[u]] = pack_bf16x8(vlo);
+                vd[dso[u] + HALF] = pack_bf16x8(vhi);
+            }
         }
     }
 }
