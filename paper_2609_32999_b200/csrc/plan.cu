@@ -292,19 +292,26 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
                 }
             }
         }
-        auto cost = [&](const AttnWork &w) {
+        // cost of an item = its (tile, 128-key step) count, kept in the item for the sorts
+        for (AttnWork &w : pl->work) {
             int c = std::min(w.step_end, steps_of(w.tile_a)) - w.step_begin;
             if (w.tile_b >= 0) c += std::min(w.step_end, steps_of(w.tile_b)) - w.step_begin;
-            return c;
-        };
+            w.cost = c;
+        }
+        auto cost = [](const AttnWork &w) { return w.cost; };
         auto sort_items = [&](std::vector<AttnWork>::iterator first_it, std::vector<AttnWork>::iterator last_it) {
             int max_cost = 1;
             for (auto it = first_it; it != last_it; ++it) max_cost = std::max(max_cost, cost(*it));
             const int band = std::max(1, max_cost / kAttnCostBands);
-            auto key = [&](const AttnWork &w) {
-                return std::make_tuple(-(cost(w) / band), pl->tiles[w.tile_a].req, w.kvh, -cost(w));
-            };
-            std::stable_sort(first_it, last_it, [&](const AttnWork &x, const AttnWork &y) { return key(x) < key(y); });
+            const AttnTile *tl = pl->tiles.data();
+            std::stable_sort(first_it, last_it, [=](const AttnWork &x, const AttnWork &y) {
+                const int bx = x.cost / band, by = y.cost / band;
+                if (bx != by) return bx > by;
+                const int rx = tl[x.tile_a].req, ry = tl[y.tile_a].req;
+                if (rx != ry) return rx < ry;
+                if (x.kvh != y.kvh) return x.kvh < y.kvh;
+                return x.cost > y.cost;
+            });
         };
         // chunks of whole requests with about equal attention cost, for the host-buffer pipeline
         std::vector<int64_t> req_cost(batch, 0);

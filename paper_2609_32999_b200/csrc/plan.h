@@ -37,7 +37,8 @@ struct AttnTile {
 // With split-KV the item covers only the 128-key steps [step_begin, step_end) and is part `part` of
 // `n_parts`; a part in which tile_a would have nothing to do names the longer tile alone.
 struct AttnWork {
-    int32_t tile_a, tile_b, kvh, step_begin, step_end, part, n_parts, pad;
+    int32_t tile_a, tile_b, kvh, step_begin, step_end, part, n_parts;
+    int32_t cost;      // (tile, step) count of the item: the host's sort key, not read by the kernel
 };
 
 // One (query tile, KV head) whose partial results have to be merged after a split-KV launch.
