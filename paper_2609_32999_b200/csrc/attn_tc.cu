@@ -18,6 +18,9 @@
 // some row's causal limit are masked.  Probabilities are taken against a reference maximum that is
 // refreshed only when a row's partial sum would exceed 2^8, so the accumulator in TMEM is rescaled
 // rarely.  Every wait is bounded (ptx::mbar_wait).
+// The kernel is persistent: one thread block per SM walks through its share of the work list, so the
+// barriers, the TMEM allocation and the tensor maps are set up once, and the next item's Q, K and V
+// loads and first S run while the softmax warps still write the previous item's result.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -63,7 +66,7 @@ constexpr uint32_t kTmemO = 256;    // O[tile] at 256 + tile * 128
 
 
 struct Barriers {
-    uint64_t q_full[2];
+    uint64_t q_full[2], q_empty[2];
     uint64_t full[kRing], empty[kRing];
     uint64_t s_full[2];
     uint64_t p_full[2];
@@ -97,11 +100,19 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return r;
 }
 
+// What one work item means for every role of the block.
+struct Item {
+    AttnWork wk;
+    AttnTile t0, t1;
+    int n_tiles, step0, n_steps0, n_steps1, n_steps, T, req_pages;
+    const int32_t *bt;
+};
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, const AttnTile *__restrict__ tiles,
-               const AttnWork *__restrict__ work, const int32_t *__restrict__ q_pos,
+               const AttnWork *__restrict__ work, int n_work, const int32_t *__restrict__ q_pos,
                const int32_t *__restrict__ page_off, const int32_t *__restrict__ pages,
                const int32_t *__restrict__ seq_len, __nv_bfloat16 *__restrict__ out, float *__restrict__ lse,
                int H_q, int g, int H_kv, int page_size, int num_pool_pages, float scale_log2, int max_parts,
@@ -116,40 +127,57 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     __shared__ __align__(8) Barriers bars;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
-    __shared__ float s_xchg[2][kRows];              // row maxima exchanged between the two column halves
+    __shared__ float s_xchg[2][kRows];              // row maxima (and, in the epilogue, row sums) exchanged between the two column halves
     __shared__ int s_flag[2][2][4][2];              // [step parity][tile][warp pair][half]
 
     // A block of a launch in which another block already gave up on a wait does not start, so a
     // stalled launch ends after one round of timeouts rather than one per block.
     if (*reinterpret_cast<volatile int *>(status) != 0) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const AttnWork wk = work[blockIdx.x];
-    const int n_tiles = wk.tile_b >= 0 ? 2 : 1;
-    const AttnTile t0 = tiles[wk.tile_a];
-    const AttnTile t1 = tiles[n_tiles == 2 ? wk.tile_b : wk.tile_a];
-    const int kvh = wk.kvh;
-    // This block covers the 128-key steps [step0, step_end) of its tiles (all of them unless the item
-    // was split); step indices below are relative to step0.
-    const int step0 = wk.step_begin;
-    const int n_steps0 = min(wk.step_end, (t0.kv_len + kStep - 1) / kStep) - step0;
-    const int n_steps1 = n_tiles == 2 ? min(wk.step_end, (t1.kv_len + kStep - 1) / kStep) - step0 : 0;
-    const int n_steps = max(n_steps0, n_steps1);
-    const int T = seq_len[t0.req];
-    const int req_pages = (T + page_size - 1) / page_size;
     const int pps = kStep / page_size;                 // pages per step: 1, 2, 4 or 8
-    const int32_t *bt = pages + page_off[t0.req];
+
+    // The block's share of the work list: round k of the grid takes items [k G, (k + 1) G), this block
+    // the b-th of them in even rounds and the b-th from the end in odd rounds (the list is sorted by
+    // cost, so the serpentine evens out the sums; blocks that run at the same time work on neighbours
+    // in the list, i.e. on the same request and KV head, and share their K/V pages in L2.  A greedy
+    // least-loaded assignment computed on the host balanced the modelled cost better and measured
+    // 0.5-2 % slower).  Every role walks the same sequence; -1 = nothing in this round.
+    const int n_rounds = (n_work + (int)gridDim.x - 1) / (int)gridDim.x;
+    auto item_index = [&](int round) {
+        const int b = (round & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;
+        const int w = round * (int)gridDim.x + b;
+        return w < n_work ? w : -1;
+    };
+    auto load_item = [&](int w) {
+        Item it;
+        it.wk = work[w];
+        it.n_tiles = it.wk.tile_b >= 0 ? 2 : 1;
+        it.t0 = tiles[it.wk.tile_a];
+        it.t1 = tiles[it.n_tiles == 2 ? it.wk.tile_b : it.wk.tile_a];
+        // the item covers the 128-key steps [step0, step_end) of its tiles (all of them unless it was
+        // split); step indices below are relative to step0
+        it.step0 = it.wk.step_begin;
+        it.n_steps0 = min(it.wk.step_end, (it.t0.kv_len + kStep - 1) / kStep) - it.step0;
+        it.n_steps1 = it.n_tiles == 2 ? min(it.wk.step_end, (it.t1.kv_len + kStep - 1) / kStep) - it.step0 : 0;
+        it.n_steps = max(it.n_steps0, it.n_steps1);
+        it.T = seq_len[it.t0.req];
+        it.req_pages = (it.T + page_size - 1) / page_size;
+        it.bt = pages + page_off[it.t0.req];
+        return it;
+    };
 
     if (tid == 0) {
         s_abort = 0;
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bars.q_full[i]), 1);
+            mbar_init(smem_u32(&bars.q_empty[i]), 1);
             mbar_init(smem_u32(&bars.s_full[i]), 1);
             mbar_init(smem_u32(&bars.p_full[i]), 2 * kRows);
             mbar_init(smem_u32(&bars.pv_done[i]), 1);
         }
         for (int i = 0; i < kRing; ++i) {
             mbar_init(smem_u32(&bars.full[i]), 1);
-            mbar_init(smem_u32(&bars.empty[i]), n_tiles);
+            mbar_init(smem_u32(&bars.empty[i]), 2);       // both MMA-issuing warps release every slot
         }
         fence_barrier_init();
     }
@@ -175,10 +203,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
         // A tile holds (128 / g) tokens x g heads = q_rows rows; when g does not divide 128 the last
-        // rows of the 128-row MMA tile are padding and are zeroed once (their results are never stored).
+        // rows of the 128-row MMA tile are padding and are zeroed once (TMA never writes them; their
+        // results are never stored).
         const int q_rows = (kRows / g) * g;
         if (q_rows < kRows) {
-            for (int q = 0; q < n_tiles; ++q)
+            for (int q = 0; q < 2; ++q)
 #pragma unroll
                 for (int hf = 0; hf < G::kHalves; ++hf) {
                     uint8_t *base = sm + kSmemQ + q * kQTileBytes + hf * kHalfBytes;
@@ -188,124 +217,157 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             fence_proxy_async_smem();
             __syncwarp();
         }
-        if (lane == 0) {
-            for (int q = 0; q < n_tiles; ++q) {
-                const AttnTile &t = q ? t1 : t0;
-                const uint32_t bar = smem_u32(&bars.q_full[q]);
-                mbar_expect_tx(bar, (uint32_t)(G::kHalves * q_rows * 128));
-#pragma unroll
-                for (int hf = 0; hf < G::kHalves; ++hf)
-                    tma_load_3d(smem_u32(sm + kSmemQ + q * kQTileBytes + hf * kHalfBytes), &tmap_q, bar, hf * 64, kvh * g, t.q_begin);
-            }
-        }
-        // ring item 2j = K of step j, item 2j+1 = V of step j
         const int steps_per_fetch = 32 / pps;
         const uint32_t page_bytes = (uint32_t)page_size * 128;     // one page inside a d half
-        for (int j0 = 0; j0 < n_steps; j0 += steps_per_fetch) {
-            // lane l holds the id of page (pps * (step0 + j0) + l); a page past the request's last one
-            // is fetched from outside the pool, which TMA fills with zeros
-            const int pi = pps * (step0 + j0) + lane;
-            const int my_page = pi < req_pages ? bt[pi] : num_pool_pages;
-            const int jn = min(steps_per_fetch, n_steps - j0);
-            for (int jj = 0; jj < jn; ++jj) {
-                int pg[8];
+        int ring_base = 0;                  // ring items issued for earlier work items
+        int q_uses[2] = {0, 0};             // how often each Q tile buffer has been filled
+        for (int round = 0; round < n_rounds; ++round) {
+            const int w = item_index(round);
+            if (w < 0) continue;
+            const Item it = load_item(w);
+            const int kvh = it.wk.kvh;
+            if (lane == 0) {
+                for (int q = 0; q < it.n_tiles; ++q) {
+                    const AttnTile &t = q ? it.t1 : it.t0;
+                    // the previous item's last S MMA has read this buffer
+                    if (q_uses[q] > 0) mbar_wait(smem_u32(&bars.q_empty[q]), (q_uses[q] - 1) & 1, abort_flag, status, 10);
+                    const uint32_t bar = smem_u32(&bars.q_full[q]);
+                    mbar_expect_tx(bar, (uint32_t)(G::kHalves * q_rows * 128));
 #pragma unroll
-                for (int k = 0; k < 8; ++k) pg[k] = __shfl_sync(0xffffffffu, my_page, (pps * jj + k) & 31);
-                if (lane == 0) {
-                    const int j = j0 + jj;
-#pragma unroll
-                    for (int kv = 0; kv < 2; ++kv) {
-                        const int item = 2 * j + kv, slot = item % kRing;
-                        mbar_wait(smem_u32(&bars.empty[slot]), ((item / kRing) & 1) ^ 1, abort_flag, status, 1 + kv);
-                        const uint32_t fb = smem_u32(&bars.full[slot]);
-                        mbar_expect_tx(fb, kSlotBytes);
-                        const uint32_t dst = smem_u32(sm + kSmemRing + slot * kSlotBytes);
-                        const CUtensorMap *tm = kv ? &tmap_v : &tmap_k;
-#pragma unroll
-                        for (int k = 0; k < 8; ++k)
-                            if (k < pps) {
-#pragma unroll
-                                for (int hf = 0; hf < G::kHalves; ++hf)
-                                    tma_load_4d(dst + hf * kHalfBytes + k * page_bytes, tm, fb, hf * 64, kvh, 0, pg[k]);
-                            }
-                    }
+                    for (int hf = 0; hf < G::kHalves; ++hf)
+                        tma_load_3d(smem_u32(sm + kSmemQ + q * kQTileBytes + hf * kHalfBytes), &tmap_q, bar, hf * 64, kvh * g, t.q_begin);
                 }
-                __syncwarp();
             }
+            for (int q = 0; q < it.n_tiles; ++q) ++q_uses[q];
+            // ring item ring_base + 2j = K of step j, + 2j + 1 = V of step j
+            for (int j0 = 0; j0 < it.n_steps; j0 += steps_per_fetch) {
+                // lane l holds the id of page (pps * (step0 + j0) + l); a page past the request's last one
+                // is fetched from outside the pool, which TMA fills with zeros
+                const int pi = pps * (it.step0 + j0) + lane;
+                const int my_page = pi < it.req_pages ? it.bt[pi] : num_pool_pages;
+                const int jn = min(steps_per_fetch, it.n_steps - j0);
+                for (int jj = 0; jj < jn; ++jj) {
+                    int pg[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) pg[k] = __shfl_sync(0xffffffffu, my_page, (pps * jj + k) & 31);
+                    if (lane == 0) {
+                        const int j = j0 + jj;
+#pragma unroll
+                        for (int kv = 0; kv < 2; ++kv) {
+                            const int item = ring_base + 2 * j + kv, slot = item % kRing;
+                            mbar_wait(smem_u32(&bars.empty[slot]), ((item / kRing) & 1) ^ 1, abort_flag, status, 1 + kv);
+                            const uint32_t fb = smem_u32(&bars.full[slot]);
+                            mbar_expect_tx(fb, kSlotBytes);
+                            const uint32_t dst = smem_u32(sm + kSmemRing + slot * kSlotBytes);
+                            const CUtensorMap *tm = kv ? &tmap_v : &tmap_k;
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+                                if (k < pps) {
+#pragma unroll
+                                    for (int hf = 0; hf < G::kHalves; ++hf)
+                                        tma_load_4d(dst + hf * kHalfBytes + k * page_bytes, tm, fb, hf * 64, kvh, 0, pg[k]);
+                                }
+                        }
+                    }
+                    __syncwarp();
+                }
+            }
+            ring_base += 2 * it.n_steps;
         }
-    } else if (warp == 9 || (warp == 10 && n_tiles == 2)) {
+    } else if (warp == 9 || warp == 10) {
         // ------------------------------------------------------------------ MMA issuers: warp 9 for
         // tile 0, warp 10 for tile 1.  Each runs its own tile's chain, so the waits of one overlap
-        // the MMAs of the other; a ring slot is free again once both have released it.
+        // the MMAs of the other; a ring slot is free again once both have released it (the warp of a
+        // tile that is absent or already finished only releases).
         constexpr uint32_t idesc_s = idesc_bf16(kRows, kStep, false);
         constexpr uint32_t idesc_o = idesc_bf16(kRows, kD, true);
         const int q = warp - 9;
-        const int my_steps = q ? n_steps1 : n_steps0;
-        const int tail_step = (T % kStep) ? T / kStep - step0 : -1;   // step holding slots past the sequence end
         const uint32_t qbase = smem_u32(sm + kSmemQ + q * kQTileBytes);
         const uint32_t tS = tmem + kTmemS + q * 128, tO = tmem + kTmemO + q * 128;
+        int ring_base = 0, step_base = 0, q_uses = 0;
 
-        auto ring_wait = [&](int item, int code) {
-            mbar_wait(smem_u32(&bars.full[item % kRing]), (item / kRing) & 1, abort_flag, status, code);
-            tc_fence_after();
-        };
-        auto issue_s = [&](int j) {                                // S[q] = Q_q K_j^T (lane 0)
-            const uint32_t kbase = smem_u32(sm + kSmemRing + ((2 * j) % kRing) * kSlotBytes);
-#pragma unroll
-            for (int k = 0; k < kD / 16; ++k) {
-                const uint64_t a = smem_desc_sw128(qbase + (k / 4) * kHalfBytes + (k % 4) * 32, 16, 1024);
-                const uint64_t b = smem_desc_sw128(kbase + (k / 4) * kHalfBytes + (k % 4) * 32, 16, 1024);
-                umma_ss(tS, a, b, idesc_s, k > 0);
-            }
-            umma_commit(smem_u32(&bars.s_full[q]));
-            umma_commit(smem_u32(&bars.empty[(2 * j) % kRing]));   // K_j no longer needed by this tile
-        };
+        for (int round = 0; round < n_rounds; ++round) {
+            const int w = item_index(round);
+            if (w < 0) continue;
+            const Item it = load_item(w);
+            const int n_steps = it.n_steps;
+            const int my_steps = q ? it.n_steps1 : it.n_steps0;
+            const int T = it.T, step0 = it.step0;
+            const int tail_step = (T % kStep) ? T / kStep - step0 : -1;   // step holding slots past the sequence end
 
-        mbar_wait(smem_u32(&bars.q_full[q]), 0, abort_flag, status, 4);
-        ring_wait(0, 3);
-        if (lane == 0) issue_s(0);
-        __syncwarp();
-        for (int j = 0; j < n_steps; ++j) {
-            ring_wait(2 * j + 1, 5);                               // V_j
-            const int vslot = (2 * j + 1) % kRing;
-            const bool more = j + 1 < n_steps;
-            if (j >= my_steps) {
-                // this tile is finished (tile 0 may need fewer steps): only release the slots
-                if (more) ring_wait(2 * j + 2, 3);
-                if (lane == 0) {
-                    mbar_arrive(smem_u32(&bars.empty[vslot]));
-                    if (more) mbar_arrive(smem_u32(&bars.empty[(2 * j + 2) % kRing]));
-                }
-                __syncwarp();
-                continue;
-            }
-            if (j == tail_step) {
-                // V rows past the end of the sequence hold whatever the page held before; their
-                // probabilities are zero, but 0 x NaN would still poison the accumulator.  (Both
-                // issuing warps may write these zeros; the values agree.)
-                uint8_t *v = sm + kSmemRing + vslot * kSlotBytes;
-                for (int r = T - (step0 + j) * kStep; r < kStep; ++r)
-                    if (lane < 8 * G::kHalves) *reinterpret_cast<uint4 *>(v + (lane >> 3) * kHalfBytes + r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
-                fence_proxy_async_smem();
-                __syncwarp();
-            }
-            const bool next_s = j + 1 < my_steps;
-            if (more) ring_wait(2 * j + 2, 3);                     // K_{j+1}
-            const uint32_t vbase = smem_u32(sm + kSmemRing + vslot * kSlotBytes);
-            mbar_wait(smem_u32(&bars.p_full[q]), j & 1, abort_flag, status, 6);
-            tc_fence_after();
-            if (lane == 0) {
+            auto ring_wait = [&](int item, int code) {
+                item += ring_base;
+                mbar_wait(smem_u32(&bars.full[item % kRing]), (item / kRing) & 1, abort_flag, status, code);
+                tc_fence_after();
+            };
+            auto slot_of = [&](int item) { return (ring_base + item) % kRing; };
+            auto issue_s = [&](int j) {                                // S[q] = Q_q K_j^T (lane 0)
+                const uint32_t kbase = smem_u32(sm + kSmemRing + slot_of(2 * j) * kSlotBytes);
 #pragma unroll
-                for (int k = 0; k < kStep / 16; ++k) {
-                    const uint64_t b = smem_desc_sw128(vbase + k * 2048, kHalfBytes, 1024);
-                    umma_ts(tO, tS + (k >> 2) * 64 + (k & 3) * 8, b, idesc_o, (j > 0) || (k > 0));
+                for (int k = 0; k < kD / 16; ++k) {
+                    const uint64_t a = smem_desc_sw128(qbase + (k / 4) * kHalfBytes + (k % 4) * 32, 16, 1024);
+                    const uint64_t b = smem_desc_sw128(kbase + (k / 4) * kHalfBytes + (k % 4) * 32, 16, 1024);
+                    umma_ss(tS, a, b, idesc_s, k > 0);
                 }
-                umma_commit(smem_u32(&bars.pv_done[q]));
-                umma_commit(smem_u32(&bars.empty[vslot]));
-                if (next_s) issue_s(j + 1);
-                else if (more) mbar_arrive(smem_u32(&bars.empty[(2 * j + 2) % kRing]));
+                umma_commit(smem_u32(&bars.s_full[q]));
+                umma_commit(smem_u32(&bars.empty[slot_of(2 * j)]));    // K_j no longer needed by this tile
+                if (j == my_steps - 1) umma_commit(smem_u32(&bars.q_empty[q]));   // the item's last read of Q
+            };
+
+            ring_wait(0, 3);
+            if (my_steps > 0) {
+                mbar_wait(smem_u32(&bars.q_full[q]), q_uses & 1, abort_flag, status, 4);
+                ++q_uses;
+                tc_fence_after();
+                if (lane == 0) issue_s(0);
+            } else if (lane == 0) {
+                mbar_arrive(smem_u32(&bars.empty[slot_of(0)]));
             }
             __syncwarp();
+            for (int j = 0; j < n_steps; ++j) {
+                ring_wait(2 * j + 1, 5);                               // V_j
+                const int vslot = slot_of(2 * j + 1);
+                const bool more = j + 1 < n_steps;
+                if (j >= my_steps) {
+                    // this tile is finished or absent: only release the slots
+                    if (more) ring_wait(2 * j + 2, 3);
+                    if (lane == 0) {
+                        mbar_arrive(smem_u32(&bars.empty[vslot]));
+                        if (more) mbar_arrive(smem_u32(&bars.empty[slot_of(2 * j + 2)]));
+                    }
+                    __syncwarp();
+                    continue;
+                }
+                if (j == tail_step) {
+                    // V rows past the end of the sequence hold whatever the page held before; their
+                    // probabilities are zero, but 0 x NaN would still poison the accumulator.  (Both
+                    // issuing warps may write these zeros; the values agree.)
+                    uint8_t *v = sm + kSmemRing + vslot * kSlotBytes;
+                    for (int r = T - (step0 + j) * kStep; r < kStep; ++r)
+                        if (lane < 8 * G::kHalves) *reinterpret_cast<uint4 *>(v + (lane >> 3) * kHalfBytes + r * 128 + (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                }
+                const bool next_s = j + 1 < my_steps;
+                if (more) ring_wait(2 * j + 2, 3);                     // K_{j+1}
+                const uint32_t vbase = smem_u32(sm + kSmemRing + vslot * kSlotBytes);
+                mbar_wait(smem_u32(&bars.p_full[q]), (step_base + j) & 1, abort_flag, status, 6);
+                tc_fence_after();
+                if (lane == 0) {
+#pragma unroll
+                    for (int k = 0; k < kStep / 16; ++k) {
+                        const uint64_t b = smem_desc_sw128(vbase + k * 2048, kHalfBytes, 1024);
+                        umma_ts(tO, tS + (k >> 2) * 64 + (k & 3) * 8, b, idesc_o, (j > 0) || (k > 0));
+                    }
+                    umma_commit(smem_u32(&bars.pv_done[q]));
+                    umma_commit(smem_u32(&bars.empty[vslot]));
+                    if (next_s) issue_s(j + 1);
+                    else if (more) mbar_arrive(smem_u32(&bars.empty[slot_of(2 * j + 2)]));
+                }
+                __syncwarp();
+            }
+            ring_base += 2 * n_steps;
+            step_base += my_steps;
         }
     }
     } else {
@@ -318,6 +380,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         const int pair = warp & 3;                     // named barrier 1 + pair joins warps w and w + 4
         const int row = tid & 127;
         const uint32_t lane_base = (uint32_t)(pair * 32) << 16;
+        int step_base[2] = {0, 0};                     // steps of each tile in earlier work items (barrier phases go on)
+
+        for (int round = 0; round < n_rounds; ++round) {
+        const int w = item_index(round);
+        if (w < 0) continue;
+        const Item it = load_item(w);
+        const int n_tiles = it.n_tiles, n_steps = it.n_steps, n_steps0 = it.n_steps0, n_steps1 = it.n_steps1;
+        const int step0 = it.step0, kvh = it.wk.kvh;
+        const AttnTile &t0 = it.t0, &t1 = it.t1;
         int tok[2], p_row[2];
         bool row_valid[2];
         float m_row[2] = {-INFINITY, -INFINITY}, l_row[2] = {0.f, 0.f};
@@ -334,8 +405,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             for (int q = 0; q < 2; ++q) {
                 if (q >= n_tiles || j >= (q ? n_steps1 : n_steps0)) continue;
                 const uint32_t tS = tmem + kTmemS + q * 128 + h * 64 + lane_base;
+                const int par = (step_base[q] + j) & 1;
                 // S_j complete; this also means P.V of step j-1 has completed (it was issued earlier)
-                mbar_wait(smem_u32(&bars.s_full[q]), j & 1, abort_flag, status, 7);
+                mbar_wait(smem_u32(&bars.s_full[q]), par, abort_flag, status, 7);
                 tc_fence_after();
                 const int key0 = (step0 + j) * kStep + h * 64;
                 const bool masked = (step0 + j) * kStep + kStep > (q ? t1.kv_full : t0.kv_full);   // a causal limit falls in this step
@@ -388,7 +460,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     stale = !(sum <= 256.f);
                 }
                 // both halves of a row must take the same decision
-                const int par = j & 1;
                 const bool warp_stale = __any_sync(0xffffffffu, stale);
                 if (lane == 0) s_flag[par][q][pair][h] = warp_stale ? 1 : 0;
                 named_sync(1 + pair, 64);
@@ -428,21 +499,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             }
         }
 
-        // epilogue: O / l -> bf16, LSE.  Both tiles' last MMAs are complete before the shared-memory
-        // ring (idle by then) is reused to add up the two partial sums of every row.
-        for (int q = 0; q < n_tiles; ++q)
-            mbar_wait(smem_u32(&bars.pv_done[q]), ((q ? n_steps1 : n_steps0) - 1) & 1, abort_flag, status, 9);
-        tc_fence_after();
-        float *l_xchg = reinterpret_cast<float *>(sm + kSmemRing);           // [tile][half][row]
-        for (int q = 0; q < n_tiles; ++q) l_xchg[(q * 2 + h) * 128 + row] = l_row[q];
-        named_sync(1 + pair, 64);
+        // epilogue of the item: O / l -> bf16, LSE.  The producer and the MMA warps are already on
+        // the next item; its first P.V needs the P these warps write after this epilogue, so the
+        // accumulators are not touched before they have been read here.
         for (int q = 0; q < n_tiles; ++q) {
             const AttnTile &t = q ? t1 : t0;
-            const float l_tot = l_row[q] + l_xchg[(q * 2 + (h ^ 1)) * 128 + row];
-            const AttnWork wke = work[blockIdx.x];     // re-read here rather than kept in registers through the loop
-            if (wke.n_parts > 1) {
+            const int my_steps = q ? n_steps1 : n_steps0;
+            mbar_wait(smem_u32(&bars.pv_done[q]), (step_base[q] + my_steps - 1) & 1, abort_flag, status, 9);
+            tc_fence_after();
+            // the two partial sums of a row meet in shared memory
+            s_xchg[h][row] = l_row[q];
+            named_sync(1 + pair, 64);
+            const float l_tot = l_row[q] + s_xchg[h ^ 1][row];
+            named_sync(1 + pair, 64);                  // s_xchg may be rewritten after this point
+            if (it.wk.n_parts > 1) {
                 // split-KV part: unnormalised accumulator, reference maximum and sum go to the workspace
-                const size_t slot = ((size_t)(q ? wke.tile_b : wke.tile_a) * H_kv + kvh) * max_parts + wke.part;
+                const size_t slot = ((size_t)(q ? it.wk.tile_b : it.wk.tile_a) * H_kv + kvh) * max_parts + it.wk.part;
                 float *po = ws_o + (slot * kRows + row) * kD + h * kOCols;
                 const uint32_t tOp = tmem + kTmemO + q * 128 + h * kOCols + lane_base;
 #pragma unroll
@@ -469,16 +541,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 if (row_valid[q]) {
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
-                        uint32_t w[4];
+                        uint32_t w4[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            w[i] = pack_bf16(__uint_as_float(o[v * 8 + 2 * i]) * inv, __uint_as_float(o[v * 8 + 2 * i + 1]) * inv);
-                        *reinterpret_cast<uint4 *>(orow + c * 32 + v * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                            w4[i] = pack_bf16(__uint_as_float(o[v * 8 + 2 * i]) * inv, __uint_as_float(o[v * 8 + 2 * i + 1]) * inv);
+                        *reinterpret_cast<uint4 *>(orow + c * 32 + v * 8) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
                     }
                 }
             }
             if (lse && row_valid[q] && h == 0)
                 lse[(size_t)(t.q_begin + tok[q]) * H_q + head] = (m_row[q] + log2f(l_tot)) * 0.6931471805599453f;
+        }
+        step_base[0] += n_steps0;
+        step_base[1] += n_steps1;
         }
     }
 
@@ -555,8 +630,10 @@ cudaError_t launch_attn_tc_d(const tessera_plan *pl, void *k_pool, void *v_pool,
     }
     const DeviceTables &d = pl->dev;
     const float scale_log2 = pl->sm_scale * 1.4426950408889634f;
-    attn_tc_kernel<D><<<(unsigned)n_work, kThreads, Geo<D>::kSmemAlloc, st>>>(
-        tq, tk, tv, d.tiles, work, d.q_pos, d.page_off, d.pages, d.seq_len,
+    // persistent: one thread block per SM (fewer when the list is shorter)
+    const unsigned grid = (unsigned)std::min<size_t>(n_work, (size_t)kNumSMs);
+    attn_tc_kernel<D><<<grid, kThreads, Geo<D>::kSmemAlloc, st>>>(
+        tq, tk, tv, d.tiles, work, (int)n_work, d.q_pos, d.page_off, d.pages, d.seq_len,
         static_cast<__nv_bfloat16 *>(out), lse, Hq, g, Hkv, ps, pl->num_pool_pages, scale_log2, pl->max_parts, d.ws_o, d.ws_ml, d.status);
     count_launch();
     if (pl->max_parts > 1) {
