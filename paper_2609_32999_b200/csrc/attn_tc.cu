@@ -94,6 +94,11 @@ __device__ __forceinline__ void add2(float &a0, float &a1, float b0, float b1) {
     asm("{\n .reg .b64 ra, rb;\n mov.b64 ra, {%0, %1};\n mov.b64 rb, {%2, %3};\n add.rn.f32x2 ra, ra, rb;\n mov.b64 {%0, %1}, ra;\n}"
         : "+f"(a0), "+f"(a1) : "f"(b0), "f"(b1));
 }
+// 32-byte store (one full sector per lane); p must be 32-byte aligned.
+__device__ __forceinline__ void stg256(void *p, const uint32_t (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -141,7 +146,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     // cost, so the serpentine evens out the sums; blocks that run at the same time work on neighbours
     // in the list, i.e. on the same request and KV head, and share their K/V pages in L2.  A greedy
     // least-loaded assignment computed on the host balanced the modelled cost better and measured
-    // 0.5-2 % slower).  Every role walks the same sequence; -1 = nothing in this round.
+    // 0.5-2 % slower; taking items off a global counter at run time measured 1-1.5 % slower on the
+    // long-context configurations).  Every role walks the same sequence; -1 = nothing in this round.
     const int n_rounds = (n_work + (int)gridDim.x - 1) / (int)gridDim.x;
     auto item_index = [&](int round) {
         const int b = (round & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;
@@ -381,6 +387,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         const int row = tid & 127;
         const uint32_t lane_base = (uint32_t)(pair * 32) << 16;
         int step_base[2] = {0, 0};                     // steps of each tile in earlier work items (barrier phases go on)
+        const bool out_aligned32 = (reinterpret_cast<uintptr_t>(out) & 31) == 0;
 
         for (int round = 0; round < n_rounds; ++round) {
         const int w = item_index(round);
@@ -539,13 +546,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 tmem_ld32(tO + c * 32, o);
                 tmem_wait_ld();
                 if (row_valid[q]) {
+                    // a row's half is 128 contiguous bytes: full 32-byte sectors when `out` allows it
+                    // (16-byte stores of 32 rows at a time kept the load/store unit busy for ~1 000 cycles per tile)
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint32_t w4[4];
+                    for (int v = 0; v < 2; ++v) {
+                        uint32_t w8[8];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            w4[i] = pack_bf16(__uint_as_float(o[v * 8 + 2 * i]) * inv, __uint_as_float(o[v * 8 + 2 * i + 1]) * inv);
-                        *reinterpret_cast<uint4 *>(orow + c * 32 + v * 8) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                        for (int i = 0; i < 8; ++i)
+                            w8[i] = pack_bf16(__uint_as_float(o[v * 16 + 2 * i]) * inv, __uint_as_float(o[v * 16 + 2 * i + 1]) * inv);
+                        if (out_aligned32) {
+                            stg256(orow + c * 32 + v * 16, w8);
+                        } else {
+                            *reinterpret_cast<uint4 *>(orow + c * 32 + v * 16) = make_uint4(w8[0], w8[1], w8[2], w8[3]);
+                            *reinterpret_cast<uint4 *>(orow + c * 32 + v * 16 + 8) = make_uint4(w8[4], w8[5], w8[6], w8[7]);
+                        }
                     }
                 }
             }

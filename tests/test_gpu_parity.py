@@ -442,3 +442,37 @@ def test_group_sizes_that_do_not_divide_the_tile(hq, hkv, D):
     w = wl.build_workload("mid", shape, [[3, wl.unit(700, "a", recompute=range(9)), wl.unit(300, "b", cached=False), 41]],
                           np.random.default_rng(hq))
     _full_check(w)
+
+
+def test_output_buffer_aligned_to_16_bytes_only():
+    """`out` need only be 16-byte aligned: the kernel's 32-byte stores fall back to 16-byte ones and
+    the result is the same, bit for bit."""
+    w = wl.config(2)
+    t = wl.make_tensors(w, device="cuda:0", seed=3)
+    plan = tb.Plan(w)
+    plan.kv_compose(t.k_pool, t.v_pool)
+    sh = w.shape
+    n = w.n_q * sh.num_q_heads * sh.head_dim
+    ref = torch.zeros(w.n_q, sh.num_q_heads, sh.head_dim, dtype=torch.bfloat16, device="cuda:0")
+    raw = torch.zeros(n + 8, dtype=torch.bfloat16, device="cuda:0")
+    off = raw[8:].view(w.n_q, sh.num_q_heads, sh.head_dim)
+    assert ref.data_ptr() % 32 == 0 and off.data_ptr() % 32 == 16
+    plan.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, ref, None)
+    plan.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, off, None)
+    torch.cuda.synchronize()
+    assert plan.status() == 0
+    assert torch.equal(ref, off) and float(ref.float().abs().sum()) > 0
+    # a non-split batch takes the direct epilogue (config 2 is split along the keys and merged afterwards)
+    w3 = wl.config(3, requests_override=4)
+    t3 = wl.make_tensors(w3, device="cuda:0", seed=4)
+    p3 = tb.Plan(w3)
+    p3.kv_compose(t3.k_pool, t3.v_pool)
+    sh3 = w3.shape
+    ref3 = torch.zeros(w3.n_q, sh3.num_q_heads, sh3.head_dim, dtype=torch.bfloat16, device="cuda:0")
+    raw3 = torch.zeros(ref3.numel() + 8, dtype=torch.bfloat16, device="cuda:0")
+    off3 = raw3[8:].view_as(ref3)
+    p3.partial_prefill_attn(t3.k_pool, t3.v_pool, t3.q, t3.k_new, t3.v_new, ref3, None)
+    p3.partial_prefill_attn(t3.k_pool, t3.v_pool, t3.q, t3.k_new, t3.v_new, off3, None)
+    torch.cuda.synchronize()
+    assert p3.status() == 0 and off3.data_ptr() % 32 == 16
+    assert torch.equal(ref3, off3) and float(ref3.float().abs().sum()) > 0
