@@ -476,3 +476,25 @@ def test_output_buffer_aligned_to_16_bytes_only():
     torch.cuda.synchronize()
     assert p3.status() == 0 and off3.data_ptr() % 32 == 16
     assert torch.equal(ref3, off3) and float(ref3.float().abs().sum()) > 0
+
+
+def test_many_uneven_items_per_thread_block():
+    """The persistent attention kernel walks many items per thread block: 240 short requests with one,
+    two or three query tiles (so single-tile items are mixed in), tiles of different lengths and keys
+    from 60 to 1 000 - every barrier phase carries over from item to item."""
+    shape = wl.ModelShape(32, 8, 128, 64, 500000.0)
+    rng = np.random.default_rng(123)
+    reqs = []
+    for r in range(240):
+        ctx = int(rng.integers(50, 900))
+        tail = int(rng.integers(1, 70))
+        reqs.append([int(rng.integers(0, 4)), wl.unit(ctx, ("u", r), recompute=(0, 1, ctx // 2)), tail])
+    w = wl.build_workload("many", shape, reqs, rng)
+    plan = tb.Plan(w, host_only=True)
+    assert plan.info.attn_kernel == 1 and plan.info.n_attn_items > 148 * 10
+    g = gu.run_layer(w, seed=99)
+    assert g.status == 0
+    gu.check_placement(g)
+    asm, _, _ = gu.check_assembled(g)
+    gu.check_untouched(g)
+    gu.check_attention(g, asm)
