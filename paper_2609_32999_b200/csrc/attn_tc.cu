@@ -6,8 +6,8 @@
 // read.  A step covers 128 keys (1, 2, 4 or 8 pages of 128, 64, 32 or 16 tokens).  Warp roles (384 threads):
 //   warps 0-7  : softmax.  All eight work on one tile at a time and alternate between the tiles;
 //                warps 0-3 own columns 0-63 of a row, warps 4-7 columns 64-127 (TMEM lane = row)
-//   warp 8     : TMA producer - Q tiles once, then K and V of every step through one ring of
-//                32 KB shared-memory slots; page ids come from the request's block table
+//   warp 8     : TMA producer - Q tiles once per item, then K and V of every step through one ring of
+//                four 32 KB shared-memory slots; page ids come from the request's block table
 //   warp 9, 10 : issue tcgen05.mma for tile 0 / tile 1 (one lane each); warp 9 owns the TMEM allocation
 //   warp 11    : idle (completes the warp group that hands its registers to the softmax warps)
 // Per tile and step:  S = Q K^T (both operands in shared memory) -> 128 fp32 TMEM columns;
@@ -38,7 +38,7 @@ using namespace ptx;
 
 constexpr int kStep = 128;         // keys per step (two pages)
 constexpr int kRows = 128;         // rows per query tile
-constexpr int kRing = 5;           // K/V ring slots
+constexpr int kRing = 4;           // K/V ring slots (two steps of look-ahead; a fifth slot measured no faster)
 constexpr int kThreads = 384;        // 8 softmax warps, producer, MMA, 2 idle warps (register donors)
 // setmaxnreg moves registers inside the pool the block got at launch (threads x registers per thread
 // under __launch_bounds__): the raised and lowered counts together must fit in it, or the raise
@@ -56,7 +56,8 @@ template <int D> struct Geo {
     static constexpr uint32_t kSlotBytes = kHalves * kHalfBytes;               // K or V of one step
     static constexpr uint32_t kSmemQ = 0;
     static constexpr uint32_t kSmemRing = kSmemQ + 2 * kQTileBytes;
-    static constexpr uint32_t kSmemTotal = kSmemRing + kRing * kSlotBytes;
+    static constexpr uint32_t kSmemStage = kSmemRing + kRing * kSlotBytes;     // one output tile (bf16), laid out like a Q tile
+    static constexpr uint32_t kSmemTotal = kSmemStage + kQTileBytes;
     static constexpr uint32_t kSmemAlloc = kSmemTotal + 1024;                  // slack for the 1024-byte alignment
 };
 
@@ -116,7 +117,8 @@ struct Item {
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-               const __grid_constant__ CUtensorMap tmap_v, const AttnTile *__restrict__ tiles,
+               const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
+               const AttnTile *__restrict__ tiles,
                const AttnWork *__restrict__ work, int n_work, const int32_t *__restrict__ q_pos,
                const int32_t *__restrict__ page_off, const int32_t *__restrict__ pages,
                const int32_t *__restrict__ seq_len, __nv_bfloat16 *__restrict__ out, float *__restrict__ lse,
@@ -195,6 +197,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         prefetch_tmap(&tmap_q);
         prefetch_tmap(&tmap_k);
         prefetch_tmap(&tmap_v);
+        prefetch_tmap(&tmap_o);
     }
     tc_fence_before();
     __syncthreads();
@@ -538,8 +541,46 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             }
             const float inv = 1.f / l_tot;
             const int head = kvh * g + row % g;
-            __nv_bfloat16 *orow = out + ((size_t)(t.q_begin + tok[q]) * H_q + head) * kD + h * kOCols;
             const uint32_t tO = tmem + kTmemO + q * 128 + h * kOCols + lane_base;
+            if (lse && row_valid[q] && h == 0)
+                lse[(size_t)(t.q_begin + tok[q]) * H_q + head] = (m_row[q] + log2f(l_tot)) * 0.6931471805599453f;
+            if (t.n_tok == kRows / g) {
+                // A full tile leaves through shared memory and one tiled bulk store per 64 columns: the tile
+                // is laid out like a Q tile (row = token * g + head, 128-byte swizzle), so the store
+                // writes whole 128-byte lines; 32 rows 256 B apart per store instruction kept the
+                // load/store unit busy three times as long.
+                uint8_t *stage = sm + G::kSmemStage;
+                if (tid == 0) bulk_wait_read();            // the previous tile's store has read the buffer
+                named_sync(5, 256);
+#pragma unroll
+                for (int c = 0; c < kOCols / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        uint32_t w4[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            w4[i] = pack_bf16(__uint_as_float(o[v * 8 + 2 * i]) * inv, __uint_as_float(o[v * 8 + 2 * i + 1]) * inv);
+                        // columns h * kOCols + c * 32 + v * 8 .. + 7 of the row: 16-byte chunk `ch` of 64-column half `hf`
+                        const int col = h * kOCols + c * 32 + v * 8;
+                        const int hf = col >> 6, ch = (col & 63) >> 3;
+                        *reinterpret_cast<uint4 *>(stage + hf * kHalfBytes + row * 128 + ((ch ^ (row & 7)) << 4)) =
+                            make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                    }
+                }
+                fence_proxy_async_smem();
+                named_sync(5, 256);
+                if (tid == 0) {
+#pragma unroll
+                    for (int hf = 0; hf < G::kHalves; ++hf)
+                        tma_store_3d(&tmap_o, smem_u32(stage + hf * kHalfBytes), hf * 64, kvh * g, t.q_begin);
+                    bulk_commit();
+                }
+                continue;
+            }
+            __nv_bfloat16 *orow = out + ((size_t)(t.q_begin + tok[q]) * H_q + head) * kD + h * kOCols;
 #pragma unroll
             for (int c = 0; c < kOCols / 32; ++c) {
                 uint32_t o[32];
@@ -563,14 +604,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     }
                 }
             }
-            if (lse && row_valid[q] && h == 0)
-                lse[(size_t)(t.q_begin + tok[q]) * H_q + head] = (m_row[q] + log2f(l_tot)) * 0.6931471805599453f;
         }
         step_base[0] += n_steps0;
         step_base[1] += n_steps1;
         }
     }
 
+    if (tid == 0) bulk_wait_all();    // the block's output stores are complete
     if (*abort_flag) {            // a wait gave up: let copies still in flight land before the block exits
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000) {}
@@ -634,8 +674,9 @@ cudaError_t launch_attn_tc_d(const tessera_plan *pl, void *k_pool, void *v_pool,
     const size_t n_work = chunk < 0 ? pl->work.size() : (size_t)(pl->chunk_work_off[chunk + 1] - pl->chunk_work_off[chunk]);
     if (n_work == 0) return cudaSuccess;
     const int Hq = pl->cfg.num_q_heads, Hkv = pl->cfg.num_kv_heads, g = Hq / Hkv, ps = pl->cfg.page_size;
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     if (!make_q_tmap(&tq, q, pl->n_q, Hq, D, g, kRows / g, err)) return cudaErrorInvalidValue;
+    if (!make_q_tmap(&to, out, pl->n_q, Hq, D, g, kRows / g, err)) return cudaErrorInvalidValue;   // `out` has the layout of q
     if (!make_pool_tmap(&tk, k_pool, pl->num_pool_pages, ps, Hkv, D, err)) return cudaErrorInvalidValue;
     if (!make_pool_tmap(&tv, v_pool, pl->num_pool_pages, ps, Hkv, D, err)) return cudaErrorInvalidValue;
     {
@@ -647,7 +688,7 @@ cudaError_t launch_attn_tc_d(const tessera_plan *pl, void *k_pool, void *v_pool,
     // persistent: one thread block per SM (fewer when the list is shorter)
     const unsigned grid = (unsigned)std::min<size_t>(n_work, (size_t)kNumSMs);
     attn_tc_kernel<D><<<grid, kThreads, Geo<D>::kSmemAlloc, st>>>(
-        tq, tk, tv, d.tiles, work, (int)n_work, d.q_pos, d.page_off, d.pages, d.seq_len,
+        tq, tk, tv, to, d.tiles, work, (int)n_work, d.q_pos, d.page_off, d.pages, d.seq_len,
         static_cast<__nv_bfloat16 *>(out), lse, Hq, g, Hkv, ps, pl->num_pool_pages, scale_log2, pl->max_parts, d.ws_o, d.ws_ml, d.status);
     count_launch();
     if (pl->max_parts > 1) {
