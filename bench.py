@@ -180,6 +180,60 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_fp8_tier(args):
+    """Side measurement, not the headline metric: the cached units of the workload sit in an e4m3 pool
+    and are expanded into the requests' bf16 pages (rotation fused), and the reverse (retain).  L2 is
+    flushed between timed launches; bytes are the algorithmic ones (1 + 2 per element either way)."""
+    import copy
+    import torch
+    from paper_2609_32999_b200 import binding as tb
+    from paper_2609_32999_b200 import workloads as wl
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    w = rank_workload(args.config, 0, args.requests, None)
+    w2 = copy.copy(w)
+    w2.num_source_pages = w.num_pool_pages
+    plan = tb.Plan(w2)
+    t = wl.make_tensors(w, layer=0, device=dev, seed=wl.BASE_SEED)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(wl.BASE_SEED)
+    shape8 = tuple(t.k_pool.shape)
+    k8 = torch.randint(0, 0x78, shape8, dtype=torch.uint8, device=dev, generator=gen)      # finite codes, both signs below
+    v8 = torch.randint(0, 0x78, shape8, dtype=torch.uint8, device=dev, generator=gen)
+    k8 |= torch.randint(0, 2, shape8, dtype=torch.uint8, device=dev, generator=gen) << 7
+    v8 |= torch.randint(0, 2, shape8, dtype=torch.uint8, device=dev, generator=gen) << 7
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def timed(fn):
+        ms = []
+        for i in range(args.warmup + args.steps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= args.warmup:
+                ms.append(a.elapsed_time(b))
+        return sum(ms) / len(ms)
+
+    launches0 = tb.launch_count()
+    ms_expand = timed(lambda: plan.kv_compose_from_fp8(k8, v8, 1 / 32, 1 / 32, t.k_pool, t.v_pool))
+    ms_retain = timed(lambda: plan.kv_retain_fp8(t.k_pool, t.v_pool, k8, v8, 1 / 32, 1 / 32))
+    elems = w.cached_tokens * w.shape.num_kv_heads * w.shape.head_dim * 2            # K and V
+    peak = measured_peaks()["hbm_gbs"]
+    line = {"metric": "fp8_tier_GBps", "unit": "GB/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+            "dtype": "e4m3 <-> bf16", "data": "synthetic",
+            "config": {"workload": w.name, "cached_tokens": int(w.cached_tokens), "l2": "flushed between launches"},
+            "expand": {"ms": ms_expand, "GBps": elems * 3 / ms_expand / 1e6, "frac_of_measured_copy": elems * 3 / ms_expand / 1e6 / peak},
+            "retain": {"ms": ms_retain, "GBps": elems * 3 / ms_retain / 1e6, "frac_of_measured_copy": elems * 3 / ms_retain / 1e6 / peak},
+            "bytes_per_launch": elems * 3, "gpu_launches": tb.launch_count() - launches0}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -195,9 +249,13 @@ def main():
                     help="residency of the units decided by a cache policy instead of 'all cached' (configs 2-4)")
     ap.add_argument("--graph", action="store_true",
                     help="replay each layer's launches from a captured CUDA graph (latency-bound small batches)")
+    ap.add_argument("--tier", default=None, choices=["fp8"],
+                    help="time the 8-bit storage tier's two kernels on the workload instead of the hot path (one GPU)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.tier == "fp8":
+        return run_fp8_tier(args)
 
     import torch
     import torch.distributed as dist
