@@ -4,8 +4,9 @@
 // One thread block works on one KV head and up to TWO query tiles of the same request (128 rows
 // each: 128/g recompute tokens x the g query heads of the group), which share every K/V page they
 // read.  A step covers 128 keys (1, 2, 4 or 8 pages of 128, 64, 32 or 16 tokens).  Warp roles (384 threads):
-//   warps 0-7  : softmax.  All eight work on one tile at a time and alternate between the tiles;
-//                warps 0-3 own columns 0-63 of a row, warps 4-7 columns 64-127 (TMEM lane = row)
+//   warps 0-7  : softmax.  All eight work on one tile at a time and alternate between the tiles; a
+//                warp owns 16 rows (TMEM lanes) and reads them as an MMA accumulator fragment, the
+//                four threads of a row in one warp - no two warps ever exchange anything
 //   warp 8     : TMA producer - Q tiles once per item, then K and V of every step through one ring of
 //                four 32 KB shared-memory slots; page ids come from the request's block table
 //   warp 9, 10 : issue tcgen05.mma for tile 0 / tile 1 (one lane each); warp 9 owns the TMEM allocation
@@ -17,7 +18,8 @@
 // for the other.  Pages past a tile's last query position are never loaded; only steps that cross
 // some row's causal limit are masked.  Probabilities are taken against a reference maximum that is
 // refreshed only when a row's partial sum would exceed 2^8, so the accumulator in TMEM is rescaled
-// rarely.  Every wait is bounded (ptx::mbar_wait).
+// rarely.  Every wait is bounded (ptx::mbar_wait).  A finished tile leaves through a shared-memory
+// output tile and a tiled bulk store.
 // The kernel is persistent: one thread block per SM walks through its share of the work list, so the
 // barriers, the TMEM allocation and the tensor maps are set up once, and the next item's Q, K and V
 // loads and first S run while the softmax warps still write the previous item's result.
@@ -95,11 +97,6 @@ __device__ __forceinline__ void add2(float &a0, float &a1, float b0, float b1) {
     asm("{\n .reg .b64 ra, rb;\n mov.b64 ra, {%0, %1};\n mov.b64 rb, {%2, %3};\n add.rn.f32x2 ra, ra, rb;\n mov.b64 {%0, %1}, ra;\n}"
         : "+f"(a0), "+f"(a1) : "f"(b0), "f"(b1));
 }
-// 32-byte store (one full sector per lane); p must be 32-byte aligned.
-__device__ __forceinline__ void stg256(void *p, const uint32_t (&w)[8]) {
-    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
-}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -130,12 +127,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     constexpr int kD = D;
     constexpr uint32_t kQTileBytes = G::kQTileBytes, kSlotBytes = G::kSlotBytes;
     constexpr uint32_t kSmemQ = G::kSmemQ, kSmemRing = G::kSmemRing;
-    constexpr int kOCols = D / 2;                      // accumulator columns per softmax thread (row, column half)
     __shared__ __align__(8) Barriers bars;
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
-    __shared__ float s_xchg[2][kRows];              // row maxima (and, in the epilogue, row sums) exchanged between the two column halves
-    __shared__ int s_flag[2][2][4][2];              // [step parity][tile][warp pair][half]
 
     // A block of a launch in which another block already gave up on a wait does not start, so a
     // stalled launch ends after one round of timeouts rather than one per block.
@@ -366,7 +360,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 #pragma unroll
                     for (int k = 0; k < kStep / 16; ++k) {
                         const uint64_t b = smem_desc_sw128(vbase + k * 2048, kHalfBytes, 1024);
-                        umma_ts(tO, tS + (k >> 2) * 64 + (k & 3) * 8, b, idesc_o, (j > 0) || (k > 0));
+                        umma_ts(tO, tS + k * 8, b, idesc_o, (j > 0) || (k > 0));   // P of keys [16k, 16k + 16): columns 8k .. 8k + 7
                     }
                     umma_commit(smem_u32(&bars.pv_done[q]));
                     umma_commit(smem_u32(&bars.empty[vslot]));
@@ -382,15 +376,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     } else {
         reg_alloc<kRegsSoftmax>();
         // ------------------------------------------------------------------ softmax + epilogue
-        // All eight warps work on ONE tile at a time and alternate between the tiles: warps 0-3 take
-        // columns 0-63 of a row, warps 4-7 columns 64-127 (warp w and w + 4 share TMEM lanes).  The
-        // two threads of a row keep identical reference maxima and separate partial sums.
-        const int h = warp >> 2;                       // column half
-        const int pair = warp & 3;                     // named barrier 1 + pair joins warps w and w + 4
-        const int row = tid & 127;
-        const uint32_t lane_base = (uint32_t)(pair * 32) << 16;
+        // All eight warps work on ONE tile at a time and alternate between the tiles.  A warp owns 16
+        // rows (TMEM lanes) with all their 128 columns - warp w the first 16 lanes of lane quarter
+        // w % 4, warp w + 4 the other 16 - and reads S in the layout of an MMA accumulator fragment:
+        // a thread holds two rows (t/4 and t/4 + 8 of the warp's 16) and, of every group of 8 columns,
+        // columns 2 (t%4) and 2 (t%4) + 1.  The four threads that share a row sit in one warp, so row
+        // maxima and sums are two shuffles away and no two warps ever have to agree on anything.
+        const int lane16 = (warp & 3) * 32 + (warp >> 2) * 16;         // first TMEM lane of this warp
+        const uint32_t lane_base = (uint32_t)lane16 << 16;
+        const int rows[2] = {lane16 + (lane >> 2), lane16 + (lane >> 2) + 8};
+        const int cq = (lane & 3) * 2;                                 // first of the thread's two columns in every group of 8
         int step_base[2] = {0, 0};                     // steps of each tile in earlier work items (barrier phases go on)
-        const bool out_aligned32 = (reinterpret_cast<uintptr_t>(out) & 31) == 0;
+        // where this thread's two bf16 of (row, column group kk) go in the swizzled output tile: rows r and
+        // r + 8 share r % 8, so one table of eight offsets serves both
+        uint32_t stage_off[8];
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) stage_off[kk] = (uint32_t)(rows[0] * 128 + ((kk ^ (rows[0] & 7)) << 4) + cq * 2);
+        auto quad_max = [](float v) {
+            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+            return fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
+        };
+        auto quad_sum = [](float v) {
+            v += __shfl_xor_sync(0xffffffffu, v, 1);
+            return v + __shfl_xor_sync(0xffffffffu, v, 2);
+        };
 
         for (int round = 0; round < n_rounds; ++round) {
         const int w = item_index(round);
@@ -399,110 +408,116 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         const int n_tiles = it.n_tiles, n_steps = it.n_steps, n_steps0 = it.n_steps0, n_steps1 = it.n_steps1;
         const int step0 = it.step0, kvh = it.wk.kvh;
         const AttnTile &t0 = it.t0, &t1 = it.t1;
-        int tok[2], p_row[2];
-        bool row_valid[2];
-        float m_row[2] = {-INFINITY, -INFINITY}, l_row[2] = {0.f, 0.f};
+        int tok[2][2], p_row[2][2];
+        bool row_valid[2][2];
+        // reference maximum (identical in the four threads of a row) and this thread's share of the row sum
+        float m_row[2][2] = {{-INFINITY, -INFINITY}, {-INFINITY, -INFINITY}}, l_row[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
             const AttnTile &t = q ? t1 : t0;
-            tok[q] = min(row / g, t.n_tok - 1);
-            row_valid[q] = row / g < t.n_tok;
-            p_row[q] = q_pos[t.q_begin + tok[q]];
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {
+                tok[q][rr] = min(rows[rr] / g, t.n_tok - 1);
+                row_valid[q][rr] = rows[rr] / g < t.n_tok;
+                p_row[q][rr] = q_pos[t.q_begin + tok[q][rr]];
+            }
         }
 
         for (int j = 0; j < n_steps; ++j) {
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 if (q >= n_tiles || j >= (q ? n_steps1 : n_steps0)) continue;
-                const uint32_t tS = tmem + kTmemS + q * 128 + h * 64 + lane_base;
+                const uint32_t tS = tmem + kTmemS + q * 128 + lane_base;
                 const int par = (step_base[q] + j) & 1;
                 // S_j complete; this also means P.V of step j-1 has completed (it was issued earlier)
                 mbar_wait(smem_u32(&bars.s_full[q]), par, abort_flag, status, 7);
                 tc_fence_after();
-                const int key0 = (step0 + j) * kStep + h * 64;
-                const bool masked = (step0 + j) * kStep + kStep > (q ? t1.kv_full : t0.kv_full);   // a causal limit falls in this step
-                const int pr = p_row[q];
+                const int key0 = (step0 + j) * kStep;
+                const bool masked = key0 + kStep > (q ? t1.kv_full : t0.kv_full);   // a causal limit falls in this step
 
                 uint32_t pk[32];
-                float sum = 0.f, mx = -INFINITY;
-                // One pass over this thread's 64 columns: the maximum (with_max) and / or the
-                // probabilities against the current reference maximum (with_exp).
+                float sum[2] = {0.f, 0.f}, mx[2] = {-INFINITY, -INFINITY};
+                // One pass over this thread's 2 x 32 scores: the row maxima (with_max) and / or the
+                // probabilities against the current reference maxima (with_exp).
                 auto pass = [&](bool with_max, bool with_exp) {
                     uint32_t s[64];
-                    tmem_ld32(tS, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-                    tmem_ld32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+                    tmem_ld_16x256b_x16(tS, s);
                     tmem_wait_ld();
                     if (masked) {
 #pragma unroll
-                        for (int i = 0; i < 64; ++i)
-                            if (key0 + i > pr) s[i] = 0xff800000u;   // -inf
+                        for (int k = 0; k < 16; ++k)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if (key0 + 8 * k + cq + (e & 1) > p_row[q][e >> 1]) s[4 * k + e] = 0xff800000u;   // -inf
                     }
                     if (with_max) {
-                        float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            mxa[i & 3] = fmaxf(mxa[i & 3], fmaxf(__uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1])));
-                        mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
+                        for (int rr = 0; rr < 2; ++rr) {
+                            float ma = -INFINITY, mb = -INFINITY;
+#pragma unroll
+                            for (int k = 0; k < 16; ++k) {
+                                ma = fmaxf(ma, __uint_as_float(s[4 * k + 2 * rr]));
+                                mb = fmaxf(mb, __uint_as_float(s[4 * k + 2 * rr + 1]));
+                            }
+                            mx[rr] = quad_max(fmaxf(ma, mb));
+                        }
                     }
                     if (with_exp) {
-                        float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+                        float sa[2][2] = {{0.f, 0.f}, {0.f, 0.f}}, sb[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
                         // a row that has seen no visible key yet (possible in a later split-KV part) keeps
                         // the reference at 0: its scores are all -inf and its probabilities 0
-                        const float neg_m = m_row[q] == -INFINITY ? 0.f : -m_row[q];
+                        const float neg_m[2] = {m_row[q][0] == -INFINITY ? 0.f : -m_row[q][0],
+                                                m_row[q][1] == -INFINITY ? 0.f : -m_row[q][1]};
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            float x0, x1;
-                            fma2(x0, x1, __uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]), scale_log2, neg_m);
-                            const float e0 = ex2(x0), e1 = ex2(x1);
-                            add2(sa[i & 3], sb[i & 3], e0, e1);
-                            pk[i] = pack_bf16(e0, e1);
-                        }
-                        sum = ((sa[0] + sb[0]) + (sa[1] + sb[1])) + ((sa[2] + sb[2]) + (sa[3] + sb[3]));
+                        for (int k = 0; k < 16; ++k)
+#pragma unroll
+                            for (int rr = 0; rr < 2; ++rr) {
+                                float x0, x1;
+                                fma2(x0, x1, __uint_as_float(s[4 * k + 2 * rr]), __uint_as_float(s[4 * k + 2 * rr + 1]), scale_log2, neg_m[rr]);
+                                const float e0 = ex2(x0), e1 = ex2(x1);
+                                add2(sa[rr][k & 1], sb[rr][k & 1], e0, e1);
+                                pk[2 * k + rr] = pack_bf16(e0, e1);      // P column 4k + t%4 of row rr
+                            }
+                        sum[0] = (sa[0][0] + sb[0][0]) + (sa[0][1] + sb[0][1]);
+                        sum[1] = (sa[1][0] + sb[1][0]) + (sa[1][1] + sb[1][1]);
                     }
                 };
 
-                // Fast path: probabilities against the current reference maximum.  While a thread's
-                // sum stays below 2^8 every probability does too and the reference is good enough;
-                // otherwise (and on the first step) the row takes the step's true maximum and redoes P.
+                // Fast path: probabilities against the current reference maxima.  While every thread's
+                // share of a row sum stays below 2^6 the row sum stays below 2^8, every probability
+                // does too and the reference is good enough; otherwise (and on the first step) the
+                // warp's rows take the step's true maxima and redo P.  The decision is per warp.
                 bool stale = true;
                 if (j > 0) {
                     pass(false, true);
-                    stale = !(sum <= 256.f);
+                    stale = !(sum[0] <= 64.f && sum[1] <= 64.f);
                 }
-                // both halves of a row must take the same decision
-                const bool warp_stale = __any_sync(0xffffffffu, stale);
-                if (lane == 0) s_flag[par][q][pair][h] = warp_stale ? 1 : 0;
-                named_sync(1 + pair, 64);
-                const bool redo = (s_flag[par][q][pair][0] | s_flag[par][q][pair][1]) != 0;
-                float factor = 1.f;
-                if (redo) {
+                float factor[2] = {1.f, 1.f};
+                if (__any_sync(0xffffffffu, stale)) {
                     pass(true, false);
-                    s_xchg[h][row] = mx;
-                    named_sync(1 + pair, 64);
-                    const float mc = fmaxf(m_row[q], fmaxf(mx, s_xchg[h ^ 1][row]) * scale_log2);
-                    if (mc != -INFINITY) {
-                        factor = ex2(m_row[q] - mc);   // 0 when the row had no visible key before
-                        m_row[q] = mc;
-                    }
-                    named_sync(1 + pair, 64);          // s_xchg may be rewritten after this point
-                    if (j > 0) {
-                        const uint32_t tO = tmem + kTmemO + q * 128 + h * kOCols + lane_base;
 #pragma unroll
-                        for (int c = 0; c < kOCols / 32; ++c) {
-                            uint32_t o[32];
-                            tmem_ld32(tO + c * 32, o);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-                            tmem_st32(tO + c * 32, o);
+                    for (int rr = 0; rr < 2; ++rr) {
+                        const float mc = fmaxf(m_row[q][rr], mx[rr] * scale_log2);
+                        if (mc != -INFINITY) {
+                            factor[rr] = ex2(m_row[q][rr] - mc);   // 0 when the row had no visible key before
+                            m_row[q][rr] = mc;
                         }
+                    }
+                    if (j > 0) {
+                        const uint32_t tO = tmem + kTmemO + q * 128 + lane_base;
+                        uint32_t o[kD / 2];
+                        if constexpr (kD == 128) tmem_ld_16x256b_x16(tO, o); else tmem_ld_16x256b_x8(tO, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < kD / 2; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor[(i >> 1) & 1]);
+                        if constexpr (kD == 128) tmem_st_16x256b_x16(tO, o); else tmem_st_16x256b_x8(tO, o);
                     }
                     pass(false, true);
                 }
-                l_row[q] = l_row[q] * factor + sum;
-                // P as bf16 over the first 32 of this thread's 64 S columns
-                tmem_st16(tS, &pk[0]);
-                tmem_st16(tS + 16, &pk[16]);
+                l_row[q][0] = l_row[q][0] * factor[0] + sum[0];
+                l_row[q][1] = l_row[q][1] * factor[1] + sum[1];
+                // P as bf16 over the first 64 columns of S: column c holds keys 2c and 2c + 1
+                tmem_st_16x128b_x16(tS, pk);
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars.p_full[q]));
@@ -517,59 +532,64 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             const int my_steps = q ? n_steps1 : n_steps0;
             mbar_wait(smem_u32(&bars.pv_done[q]), (step_base[q] + my_steps - 1) & 1, abort_flag, status, 9);
             tc_fence_after();
-            // the two partial sums of a row meet in shared memory
-            s_xchg[h][row] = l_row[q];
-            named_sync(1 + pair, 64);
-            const float l_tot = l_row[q] + s_xchg[h ^ 1][row];
-            named_sync(1 + pair, 64);                  // s_xchg may be rewritten after this point
+            const float l_tot[2] = {quad_sum(l_row[q][0]), quad_sum(l_row[q][1])};
+            const uint32_t tO = tmem + kTmemO + q * 128 + lane_base;
+            uint32_t o[kD / 2];
             if (it.wk.n_parts > 1) {
                 // split-KV part: unnormalised accumulator, reference maximum and sum go to the workspace
                 const size_t slot = ((size_t)(q ? it.wk.tile_b : it.wk.tile_a) * H_kv + kvh) * max_parts + it.wk.part;
-                float *po = ws_o + (slot * kRows + row) * kD + h * kOCols;
-                const uint32_t tOp = tmem + kTmemO + q * 128 + h * kOCols + lane_base;
+                if constexpr (kD == 128) tmem_ld_16x256b_x16(tO, o); else tmem_ld_16x256b_x8(tO, o);
+                tmem_wait_ld();
 #pragma unroll
-                for (int c = 0; c < kOCols / 32; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tOp + c * 32, o);
-                    tmem_wait_ld();
+                for (int rr = 0; rr < 2; ++rr) {
+                    float *po = ws_o + (slot * kRows + rows[rr]) * kD + cq;
 #pragma unroll
-                    for (int v = 0; v < 8; ++v)
-                        *reinterpret_cast<uint4 *>(po + c * 32 + v * 4) = make_uint4(o[v * 4], o[v * 4 + 1], o[v * 4 + 2], o[v * 4 + 3]);
+                    for (int k = 0; k < kD / 8; ++k)
+                        *reinterpret_cast<uint2 *>(po + 8 * k) = make_uint2(o[4 * k + 2 * rr], o[4 * k + 2 * rr + 1]);
+                    if ((lane & 3) == 0) ws_ml[slot * kRows + rows[rr]] = make_float2(m_row[q][rr], l_tot[rr]);
                 }
-                if (h == 0) ws_ml[slot * kRows + row] = make_float2(m_row[q], l_tot);
                 continue;
             }
-            const float inv = 1.f / l_tot;
-            const int head = kvh * g + row % g;
-            const uint32_t tO = tmem + kTmemO + q * 128 + h * kOCols + lane_base;
-            if (lse && row_valid[q] && h == 0)
-                lse[(size_t)(t.q_begin + tok[q]) * H_q + head] = (m_row[q] + log2f(l_tot)) * 0.6931471805599453f;
-            if (t.n_tok == kRows / g) {
-                // A full tile leaves through shared memory and one tiled bulk store per 64 columns: the tile
-                // is laid out like a Q tile (row = token * g + head, 128-byte swizzle), so the store
-                // writes whole 128-byte lines; 32 rows 256 B apart per store instruction kept the
-                // load/store unit busy three times as long.
-                uint8_t *stage = sm + G::kSmemStage;
+            const float inv[2] = {__frcp_rn(l_tot[0]), __frcp_rn(l_tot[1])};
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr)
+                if (lse && row_valid[q][rr] && (lane & 3) == 0)
+                    lse[(size_t)(t.q_begin + tok[q][rr]) * H_q + kvh * g + rows[rr] % g] =
+                        (m_row[q][rr] + log2f(l_tot[rr])) * 0.6931471805599453f;
+            const bool full_tile = t.n_tok == kRows / g;
+            uint8_t *stage = sm + G::kSmemStage;
+            if (full_tile) {
+                // A full tile leaves through shared memory and one tiled bulk store per 64 columns: the
+                // tile is laid out like a Q tile (row = token * g + head, 128-byte swizzle), so the
+                // store writes whole 128-byte lines.
                 if (tid == 0) bulk_wait_read();            // the previous tile's store has read the buffer
                 named_sync(5, 256);
+            }
+            if constexpr (kD == 128) tmem_ld_16x256b_x16(tO, o); else tmem_ld_16x256b_x8(tO, o);
+            tmem_wait_ld();
+            if (full_tile) {
 #pragma unroll
-                for (int c = 0; c < kOCols / 32; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tO + c * 32, o);
-                    tmem_wait_ld();
+                for (int rr = 0; rr < 2; ++rr)
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint32_t w4[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            w4[i] = pack_bf16(__uint_as_float(o[v * 8 + 2 * i]) * inv, __uint_as_float(o[v * 8 + 2 * i + 1]) * inv);
-                        // columns h * kOCols + c * 32 + v * 8 .. + 7 of the row: 16-byte chunk `ch` of 64-column half `hf`
-                        const int col = h * kOCols + c * 32 + v * 8;
-                        const int hf = col >> 6, ch = (col & 63) >> 3;
-                        *reinterpret_cast<uint4 *>(stage + hf * kHalfBytes + row * 128 + ((ch ^ (row & 7)) << 4)) =
-                            make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                    for (int k = 0; k < kD / 8; ++k) {
+                        // columns 8k + cq, + 1 of row rows[rr]: 16-byte chunk k % 8 of 64-column half k / 8
+                        float y0, y1;
+                        fma2(y0, y1, __uint_as_float(o[4 * k + 2 * rr]), __uint_as_float(o[4 * k + 2 * rr + 1]), inv[rr], 0.f);
+                        *reinterpret_cast<uint32_t *>(stage + (k >> 3) * kHalfBytes + rr * (8 * 128) + stage_off[k & 7]) = pack_bf16(y0, y1);
                     }
+            } else {
+                // a request's last, partly filled tile: 4-byte stores straight to `out`
+#pragma unroll
+                for (int rr = 0; rr < 2; ++rr) {
+                    if (!row_valid[q][rr]) continue;
+                    __nv_bfloat16 *orow = out + ((size_t)(t.q_begin + tok[q][rr]) * H_q + kvh * g + rows[rr] % g) * kD + cq;
+#pragma unroll
+                    for (int k = 0; k < kD / 8; ++k)
+                        *reinterpret_cast<uint32_t *>(orow + 8 * k) =
+                            pack_bf16(__uint_as_float(o[4 * k + 2 * rr]) * inv[rr], __uint_as_float(o[4 * k + 2 * rr + 1]) * inv[rr]);
                 }
+            }
+            if (full_tile) {
                 fence_proxy_async_smem();
                 named_sync(5, 256);
                 if (tid == 0) {
@@ -577,31 +597,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     for (int hf = 0; hf < G::kHalves; ++hf)
                         tma_store_3d(&tmap_o, smem_u32(stage + hf * kHalfBytes), hf * 64, kvh * g, t.q_begin);
                     bulk_commit();
-                }
-                continue;
-            }
-            __nv_bfloat16 *orow = out + ((size_t)(t.q_begin + tok[q]) * H_q + head) * kD + h * kOCols;
-#pragma unroll
-            for (int c = 0; c < kOCols / 32; ++c) {
-                uint32_t o[32];
-                tmem_ld32(tO + c * 32, o);
-                tmem_wait_ld();
-                if (row_valid[q]) {
-                    // a row's half is 128 contiguous bytes: full 32-byte sectors when `out` allows it
-                    // (16-byte stores of 32 rows at a time kept the load/store unit busy for ~1 000 cycles per tile)
-#pragma unroll
-                    for (int v = 0; v < 2; ++v) {
-                        uint32_t w8[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            w8[i] = pack_bf16(__uint_as_float(o[v * 16 + 2 * i]) * inv, __uint_as_float(o[v * 16 + 2 * i + 1]) * inv);
-                        if (out_aligned32) {
-                            stg256(orow + c * 32 + v * 16, w8);
-                        } else {
-                            *reinterpret_cast<uint4 *>(orow + c * 32 + v * 16) = make_uint4(w8[0], w8[1], w8[2], w8[3]);
-                            *reinterpret_cast<uint4 *>(orow + c * 32 + v * 16 + 8) = make_uint4(w8[4], w8[5], w8[6], w8[7]);
-                        }
-                    }
                 }
             }
         }
