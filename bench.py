@@ -28,7 +28,7 @@ if ROOT not in sys.path:
 # DRAM traffic per launch of the two main kernels on config 4, from the ncu capture summarised under
 # profiles/ (one request captured; a full launch is `requests` times that, traffic grows with the
 # number of requests because requests share nothing).  Bytes per request per launch.
-NCU_TRAFFIC_PER_REQUEST_C4 = {"attn": 250.8e6 + 11.7e6, "gather": 134.5e6 + 79.4e6}
+NCU_TRAFFIC_PER_REQUEST_C4 = {"attn": 253.5e6 + 14.7e6, "gather": 134.5e6 + 79.4e6}
 
 METRIC = "composed_prefill_tokens_per_s_per_layer"
 UNIT = "tokens/s"
