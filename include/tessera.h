@@ -122,8 +122,7 @@ typedef struct tessera_plan_info {
     int32_t n_rope_rows;        /* distinct shift amounts in the cos/sin table                  */
     int32_t n_gather_items;     /* thread blocks of the gather kernel                           */
     int32_t n_attn_items;       /* (q tile, kv head) work items of the attention kernel         */
-    int32_t attn_kernel;        /* 0 = generic SIMT kernel, 1 = tcgen05 kernel (page_size 16, 32, 64
-                                   or 128; any H_q/H_kv up to 16)                                         */
+    int32_t attn_kernel;        /* always 1: the tcgen05 kernel covers every shape the plan accepts      */
 } tessera_plan_info;
 
 /*

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtessera.so")
-SOURCES = ["api.cu", "plan.cu", "gather_rope.cu", "kv_fp8.cu", "attn_simt.cu", "attn_tc.cu",
+SOURCES = ["api.cu", "plan.cu", "gather_rope.cu", "kv_fp8.cu", "attn_tc.cu",
            "rope_shift_static.cu", "selftest.cu"]
 EXTRA = os.environ.get("TESSERA_NVCC_EXTRA", "").split()     # extra nvcc flags for experiments
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

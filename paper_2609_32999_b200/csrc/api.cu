@@ -120,13 +120,9 @@ bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) !=
 int32_t attention(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, const void *k_new,
                   const void *v_new, void *out, float *lse, int chunk, cudaStream_t st) {
     TS_CUDA(launch_scatter_fresh(pl, k_pool, v_pool, k_new, v_new, chunk, st));
-    if (pl->attn_kernel == 1) {
-        std::string err;
-        cudaError_t e = launch_attn_tc(pl, k_pool, v_pool, q, out, lse, chunk, st, &err);
-        if (e != cudaSuccess) return set_error(TESSERA_CUDA_ERROR, "tcgen05 attention launch: " + err + " / " + cudaGetErrorString(e));
-    } else {
-        TS_CUDA(launch_attn_simt(pl, k_pool, v_pool, q, out, lse, chunk, st));
-    }
+    std::string err;
+    cudaError_t e = launch_attn_tc(pl, k_pool, v_pool, q, out, lse, chunk, st, &err);
+    if (e != cudaSuccess) return set_error(TESSERA_CUDA_ERROR, "tcgen05 attention launch: " + err + " / " + cudaGetErrorString(e));
     return TESSERA_OK;
 }
 
@@ -231,7 +227,7 @@ int32_t tessera_plan_get_info(const tessera_plan *pl, tessera_plan_info *info) {
     info->attn_flops = 4LL * pl->cfg.head_dim * pl->cfg.num_q_heads * pl->qk_pairs;
     info->n_rope_rows = (int32_t)pl->rope_delta.size();
     info->n_gather_items = (int32_t)pl->items.size();
-    info->n_attn_items = pl->attn_kernel == 1 ? (int32_t)pl->work.size() : (int32_t)(pl->n_q * pl->cfg.num_kv_heads);
+    info->n_attn_items = (int32_t)pl->work.size();
     info->attn_kernel = pl->attn_kernel;
     return TESSERA_OK;
 }

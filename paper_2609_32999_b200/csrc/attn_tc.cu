@@ -3,7 +3,7 @@
 //
 // One thread block works on one KV head and up to TWO query tiles of the same request (128 rows
 // each: 128/g recompute tokens x the g query heads of the group), which share every K/V page they
-// read.  A step covers 128 keys (1, 2, 4 or 8 pages of 128, 64, 32 or 16 tokens).  Warp roles (384 threads):
+// read.  A step covers 128 keys (1, 2, 4, 8 or 16 pages of 128, 64, 32, 16 or 8 tokens).  Warp roles (384 threads):
 //   warps 0-7  : softmax.  All eight work on one tile at a time and alternate between the tiles; a
 //                warp owns 16 rows (TMEM lanes) and reads them as an MMA accumulator fragment, the
 //                four threads of a row in one warp - no two warps ever exchange anything
@@ -111,7 +111,9 @@ struct Item {
     const int32_t *bt;
 };
 
-template <int D>
+// kMaxPages: most pages a 128-key step can consist of in this instantiation - 8 (pages of 16 tokens or
+// more) or 16 (pages of 8 tokens); the wider producer loop is kept out of the common instantiation.
+template <int D, int kMaxPages>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
@@ -135,7 +137,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     // stalled launch ends after one round of timeouts rather than one per block.
     if (*reinterpret_cast<volatile int *>(status) != 0) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int pps = kStep / page_size;                 // pages per step: 1, 2, 4 or 8
+    const int pps = kStep / page_size;                 // pages per step: 1, 2, 4, 8 or 16
 
     // The block's share of the work list: round k of the grid takes items [k G, (k + 1) G), this block
     // the b-th of them in even rounds and the b-th from the end in odd rounds (the list is sorted by
@@ -250,9 +252,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 const int my_page = pi < it.req_pages ? it.bt[pi] : num_pool_pages;
                 const int jn = min(steps_per_fetch, it.n_steps - j0);
                 for (int jj = 0; jj < jn; ++jj) {
-                    int pg[8];
+                    int pg[kMaxPages];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) pg[k] = __shfl_sync(0xffffffffu, my_page, (pps * jj + k) & 31);
+                    for (int k = 0; k < kMaxPages; ++k) pg[k] = __shfl_sync(0xffffffffu, my_page, (pps * jj + k) & 31);
                     if (lane == 0) {
                         const int j = j0 + jj;
 #pragma unroll
@@ -264,7 +266,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                             const uint32_t dst = smem_u32(sm + kSmemRing + slot * kSlotBytes);
                             const CUtensorMap *tm = kv ? &tmap_v : &tmap_k;
 #pragma unroll
-                            for (int k = 0; k < 8; ++k)
+                            for (int k = 0; k < kMaxPages; ++k)
                                 if (k < pps) {
 #pragma unroll
                                     for (int hf = 0; hf < G::kHalves; ++hf)
@@ -662,7 +664,7 @@ attn_combine_kernel(const CombineItem *__restrict__ items, const AttnTile *__res
     if (lse && lane == 0) lse[(size_t)tok * H_q + head] = (m + log2f(l)) * 0.6931471805599453f;
 }
 
-template <int D>
+template <int D, int kMaxPages>
 cudaError_t launch_attn_tc_d(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
                              float *lse, int chunk, cudaStream_t st, std::string *err) {
     const AttnWork *work = chunk < 0 ? pl->dev.work : pl->dev.work_chunked + pl->chunk_work_off[chunk];
@@ -675,14 +677,14 @@ cudaError_t launch_attn_tc_d(const tessera_plan *pl, void *k_pool, void *v_pool,
     if (!make_pool_tmap(&tk, k_pool, pl->num_pool_pages, ps, Hkv, D, err)) return cudaErrorInvalidValue;
     if (!make_pool_tmap(&tv, v_pool, pl->num_pool_pages, ps, Hkv, D, err)) return cudaErrorInvalidValue;
     {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Geo<D>::kSmemAlloc);
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D, kMaxPages>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Geo<D>::kSmemAlloc);
         if (e != cudaSuccess) { *err = "cudaFuncSetAttribute(shared memory)"; return e; }
     }
     const DeviceTables &d = pl->dev;
     const float scale_log2 = pl->sm_scale * 1.4426950408889634f;
     // persistent: one thread block per SM (fewer when the list is shorter)
     const unsigned grid = (unsigned)std::min<size_t>(n_work, (size_t)kNumSMs);
-    attn_tc_kernel<D><<<grid, kThreads, Geo<D>::kSmemAlloc, st>>>(
+    attn_tc_kernel<D, kMaxPages><<<grid, kThreads, Geo<D>::kSmemAlloc, st>>>(
         tq, tk, tv, to, d.tiles, work, (int)n_work, d.q_pos, d.page_off, d.pages, d.seq_len,
         static_cast<__nv_bfloat16 *>(out), lse, Hq, g, Hkv, ps, pl->num_pool_pages, scale_log2, pl->max_parts, d.ws_o, d.ws_ml, d.status);
     count_launch();
@@ -706,12 +708,15 @@ cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, c
                            float *lse, int chunk, cudaStream_t st, std::string *err) {
     if (pl->n_q == 0 || pl->work.empty()) return cudaSuccess;
     const int D = pl->cfg.head_dim, ps = pl->cfg.page_size, g = pl->cfg.num_q_heads / pl->cfg.num_kv_heads;
-    if ((D != 64 && D != 128) || (ps != 16 && ps != 32 && ps != 64 && ps != 128) || g > 16) {
+    if ((D != 64 && D != 128) || (ps != 8 && ps != 16 && ps != 32 && ps != 64 && ps != 128) || g > 16) {
         *err = "shape outside the tcgen05 kernel's range";
         return cudaErrorNotSupported;
     }
-    return D == 128 ? launch_attn_tc_d<128>(pl, k_pool, v_pool, q, out, lse, chunk, st, err)
-                    : launch_attn_tc_d<64>(pl, k_pool, v_pool, q, out, lse, chunk, st, err);
+    if (ps == 8)
+        return D == 128 ? launch_attn_tc_d<128, 16>(pl, k_pool, v_pool, q, out, lse, chunk, st, err)
+                        : launch_attn_tc_d<64, 16>(pl, k_pool, v_pool, q, out, lse, chunk, st, err);
+    return D == 128 ? launch_attn_tc_d<128, 8>(pl, k_pool, v_pool, q, out, lse, chunk, st, err)
+                    : launch_attn_tc_d<64, 8>(pl, k_pool, v_pool, q, out, lse, chunk, st, err);
 }
 
 }  // namespace tessera

@@ -24,9 +24,8 @@ cudaError_t launch_rope_fresh(const tessera_plan *pl, void *q, void *k_new, cuda
 // k_new / v_new / q / out / lse always point at row 0 of the whole batch.
 cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_pool, const void *k_new,
                                  const void *v_new, int chunk, cudaStream_t st);
-cudaError_t launch_attn_simt(const tessera_plan *pl, const void *k_pool, const void *v_pool, const void *q,
-                             void *out, float *lse, int chunk, cudaStream_t st);
-// tcgen05 path; returns cudaErrorNotSupported when the plan's shape is outside its range.
+// tcgen05 attention; returns cudaErrorNotSupported when the plan's shape is outside its range (the plan
+// builder accepts no such shape).
 cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
                            float *lse, int chunk, cudaStream_t st, std::string *err);
 

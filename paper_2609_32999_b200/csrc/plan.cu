@@ -227,9 +227,8 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
 
     // ---- attention work list: tiles of consecutive recompute rows of one request
     const int g = Hq / Hkv;
-    pl->attn_kernel = 0;
     pl->tile_tokens = kAttnTileRows / g;
-    if (kHaveTensorCoreKernel && (B == 16 || B == 32 || B == 64 || B == 128)) pl->attn_kernel = 1;
+    pl->attn_kernel = 1;       // the tcgen05 kernel covers every accepted shape (page size 8..128, head_dim 64 / 128, g <= 16)
     pl->tiles.clear();
     for (int r = 0; r < batch; ++r)
         for (int j0 = d->recompute_off[r]; j0 < d->recompute_off[r + 1]; j0 += pl->tile_tokens) {
@@ -316,11 +315,6 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
         // chunks of whole requests with about equal attention cost, for the host-buffer pipeline
         std::vector<int64_t> req_cost(batch, 0);
         for (const AttnWork &w : pl->work) req_cost[pl->tiles[w.tile_a].req] += cost(w);
-        if (pl->attn_kernel != 1)      // generic kernel: cost = (query, key) pairs of the request
-            for (int r = 0; r < batch; ++r) {
-                req_cost[r] = 0;
-                for (int j = d->recompute_off[r]; j < d->recompute_off[r + 1]; ++j) req_cost[r] += d->recompute_pos[j] + 1;
-            }
         int64_t total_cost = 0;
         for (int64_t c : req_cost) total_cost += c;
         const int n_chunks = std::max(1, std::min(batch, kHostChunks));

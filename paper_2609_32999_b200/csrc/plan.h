@@ -13,7 +13,6 @@ namespace tessera {
 
 constexpr int kGatherItemTokens = 32;   // token rows per thread block of the gather kernel
 constexpr int kAttnTileRows = 128;      // query rows (tokens x grouped heads) per tcgen05 tile
-constexpr bool kHaveTensorCoreKernel = true;
 constexpr int kNumSMs = 148;              // thread blocks of the persistent attention kernel: one per SM of a B200
 constexpr int kSplitTargetBlocks = 148;  // split-KV aims at about this many thread blocks when a batch has fewer items
 constexpr int kSplitMinSteps = 4;        // never split below this many 128-key steps per part

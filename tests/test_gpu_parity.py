@@ -373,7 +373,7 @@ def test_interleaved_rope_pairing(shape):
                                    wl.ModelShape(8, 4, 128, 32, 500000.0), wl.ModelShape(32, 8, 128, 64, 500000.0)])
 def test_degenerate_layouts(shape):
     """One-token requests, one-token units, a unit that exactly fills a page, a request made of a single
-    recomputed token, page sizes 8 / 32 / 128 (generic kernel) and 64 (tensor-core kernel)."""
+    recomputed token, page sizes 8 / 32 / 64 / 128."""
     B = shape.page_size
     reqs = [[1],                                                        # a single fresh token
             [wl.unit(1, "one", cached_pos=3), 1],                       # one cached token + one fresh
@@ -414,9 +414,9 @@ def test_sharp_softmax_with_frequent_reference_refresh():
     assert e.max() <= gu.MAX_ABS and e.mean() <= gu.MEAN_ABS
 
 
-@pytest.mark.parametrize("page", [16, 32, 128])
+@pytest.mark.parametrize("page", [8, 16, 32, 128])
 def test_tensor_core_path_with_other_page_sizes(page):
-    """A 128-key step is 8, 4 or 1 pages instead of 2."""
+    """A 128-key step is 16, 8, 4 or 1 pages instead of 2."""
     shape = wl.ModelShape(32, 8, 128, page, 500000.0)
     g, _ = _full_check(wl.adversarial(seed=40 + page, shape=shape))
     assert g.plan.info.attn_kernel == 1
