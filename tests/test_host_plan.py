@@ -46,6 +46,14 @@ def test_host_only_plan_refuses_device_calls():
     with pytest.raises(tb.TesseraError) as e:
         plan.kv_compose(None, None, stream=0)
     assert e.value.status == tb.INVALID_ARG and "HOST_ONLY" in str(e.value)
+    for call in (lambda: plan.kv_compose_from_fp8(None, None, 1.0, 1.0, None, None, stream=0),
+                 lambda: plan.kv_retain_fp8(None, None, None, None, 1.0, 1.0, stream=0),
+                 lambda: plan.kv_compose_from(None, None, None, None, stream=0),
+                 lambda: plan.rope_shift(None, stream=0),
+                 lambda: plan.partial_prefill_attn(None, None, None, None, None, None, None, stream=0)):
+        with pytest.raises(tb.TesseraError) as e:
+            call()
+        assert e.value.status == tb.INVALID_ARG
 
 
 def _base():
