@@ -240,8 +240,10 @@ TESSERA_API int32_t tessera_rope_fresh(const tessera_plan *plan, void *q, void *
  *      belong to this request only.  Skipped when k_new and v_new are both NULL.
  *   2. out[j][h] = softmax(sm_scale * q[j][h] . K[0..p_j][h/g]) . V[0..p_j][h/g] over the request's
  *      assembled pages, p_j = recompute_pos[j]; bf16 inputs, fp32 accumulation and softmax.
- *   q, out: device [n_q][H_q][D] bf16.  lse: device [n_q][H_q] fp32 natural-log sum of exponentials,
- *   nullable.
+ *   q, out: device [n_q][H_q][D] bf16, 16-byte aligned (both are addressed through tiled bulk copies).
+ *   lse: device [n_q][H_q] fp32 natural-log sum of exponentials, nullable.
+ *   One persistent kernel (one thread block per SM) runs the whole batch; a batch too small to fill the
+ *   GPU is split along the keys and merged by a second kernel.
  */
 TESSERA_API int32_t tessera_partial_prefill_attn(const tessera_plan *plan, void *k_pool, void *v_pool,
                                      const void *q, const void *k_new, const void *v_new,
