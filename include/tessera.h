@@ -103,6 +103,18 @@ typedef struct tessera_compose_desc {
     const int32_t *unit_target_stride;  /* [n_units] 1 (default): token i is rotated for position
                                            target_pos + i; 0: every token is rotated for position
                                            target_pos (with target_pos = 0: written without rotation)     */
+    /* Optional (NULL = nothing is kept): units that tessera_extend_write CAPTURES for the cache while it
+       writes the request's fresh rows (Sec. 6.1: the forward path captures pre-RoPE keys and values;
+       Sec. 5.3: the miss prefill keeps the same unrotated copy for the cache). */
+    const int32_t *unit_retain_page_off;/* [n_units+1] CSR into unit_retain_pages.  A non-empty range marks a
+                                           unit to keep: every one of its tokens must be a recompute row (an
+                                           uncached unit, or a cached one recomputed in full), and the range
+                                           must hold ceil(len / page_size) pages.  Token i of the unit lands in
+                                           slot pages[i / page_size] * page_size + i % page_size               */
+    const int32_t *unit_retain_pages;   /* cache page ids, all distinct                                          */
+    int32_t retain_pool_pages;          /* 0 (default): the cache pages are pages of the destination pool itself
+                                           (k_cache = k_pool) and must be neither source nor destination pages of
+                                           this batch.  > 0: they index a separate cache pool of this many pages */
 } tessera_compose_desc;
 
 typedef struct tessera_plan tessera_plan;
@@ -123,6 +135,11 @@ typedef struct tessera_plan_info {
     int32_t n_gather_items;     /* thread blocks of the gather kernel                           */
     int32_t n_attn_items;       /* (q tile, kv head) work items of the attention kernel         */
     int32_t attn_kernel;        /* always 1: the tcgen05 kernel covers every shape the plan accepts      */
+    int64_t retained_tokens;    /* recompute rows that tessera_extend_write also writes to cache pages      */
+    int64_t attn_mma_pairs;     /* (query row, key) products the attention kernel issues to the tensor cores:
+                                   128 rows x 128 keys per (tile, step), summed over the work list.  The
+                                   algorithmic count is qk_pairs * H_q; the difference is padding rows, keys
+                                   above a row's causal limit inside a tile, and the ragged last step       */
 } tessera_plan_info;
 
 /*
@@ -234,6 +251,30 @@ TESSERA_API int32_t tessera_rope_shift(const tessera_plan *plan, void *k_pool, v
 TESSERA_API int32_t tessera_rope_fresh(const tessera_plan *plan, void *q, void *k_new, void *stream);
 
 /*
+ * The write side of the extend pass in ONE pass over the fresh rows (Sec. 5.3 "Completing prefill";
+ * Sec. 6.1: "the forward path captures pre-RoPE keys and values").  The caller hands over the layer's
+ * projections BEFORE rotation.  For every recompute row j at position p_j = recompute_pos[j]:
+ *   - k_new_raw[j] is read once; rotated for p_j it is written to the row's destination slot in
+ *     k_pool (overriding a cached value: recomputed states belong to this request), and - when the
+ *     row belongs to a unit marked by desc.unit_retain_page_off - its UNROTATED bits are also written
+ *     to the unit's cache page in k_cache;
+ *   - v_new[j] is copied to the destination slot in v_pool and, for a retained unit, to v_cache
+ *     (bit copies: values carry no rotation, Sec. 2.2);
+ *   - q[j] (nullable) is rotated for p_j in place.
+ * Angle, cosine and sine are evaluated in fp64 on the device and used as fp32; fp32 math, one
+ * round-to-nearest-even to bf16; a row at position 0 comes through bit for bit.  The captured unit is
+ * position-free: a later plan reuses it as a cached unit with unit_cached_stride = 0.
+ *   q [n_q][H_q][D], k_new_raw / v_new [n_q][H_kv][D]: device bf16, 16-byte aligned; k_new_raw and v_new
+ *   are never written.  k_cache / v_cache: device pools in the pool layout with retain_pool_pages pages
+ *   (or k_pool / v_pool themselves when retain_pool_pages is 0); nullable when the plan retains nothing.
+ * After this call tessera_partial_prefill_attn is called with k_new = v_new = NULL (its own scatter is
+ * then skipped) and the rotated q.  One kernel launch; nothing is allocated.
+ */
+TESSERA_API int32_t tessera_extend_write(const tessera_plan *plan, void *k_pool, void *v_pool, void *q,
+                                         const void *k_new_raw, const void *v_new, void *k_cache, void *v_cache,
+                                         void *stream);
+
+/*
  * Completing prefill (Sec. 5.3): the extend pass restricted to the recompute rows.
  *   1. writes k_new / v_new (device, [n_q][H_kv][D], keys already rotated at their target
  *      positions) into the rows' destination slots, overriding cached values - recomputed states
@@ -269,23 +310,30 @@ TESSERA_API int32_t tessera_composed_prefill_host(tessera_plan *plan, void *k_po
  * the library image, which every device that loads the library holds until the process exits.
  *
  * Rotates, in place, row slots[i] of k_pool (device, pool layout above) by shifts[slot_shift[i]]
- * positions, with the arithmetic of tessera_rope_shift (cos/sin in fp64 stored as fp32, fp32 math,
- * one round-to-nearest-even to bf16; a shift of 0 leaves the bits unchanged).
- *   cfg        host: head_dim, num_kv_heads, rope_theta / inv_freq, rope_pairing are read
- *   slots      device [n_slots] pool slot ids (page * page_size + offset); each listed once
- *   slot_shift device [n_slots] index into shifts; entries outside [0, n_shifts) are skipped
- *   shifts     host   [n_shifts] shift amounts; n_shifts <= TESSERA_STATIC_MAX_SHIFTS, otherwise
- *              TESSERA_UNSUPPORTED_SHAPE and nothing is launched
+ * positions, with the arithmetic of tessera_rope_shift (angle, cosine and sine in fp64 stored as
+ * fp32, fp32 math, one round-to-nearest-even to bf16; a shift of 0 leaves the bits unchanged).
+ *   cfg            host: head_dim (64 or 128), num_kv_heads and rope_theta / inv_freq are read.
+ *                  rope_pairing must be 0: only half-split pairs (m, m + D/2) are supported here;
+ *                  rope_pairing = 1 is refused with TESSERA_UNSUPPORTED_SHAPE
+ *   num_pool_slots rows in k_pool (num_pool_pages * page_size): the bound every listed slot is checked
+ *                  against on the device
+ *   slots          device [n_slots] pool slot ids (page * page_size + offset); each listed once.
+ *                  An id outside [0, num_pool_slots) is skipped: that row is neither read nor written
+ *   slot_shift     device [n_slots] index into shifts; entries outside [0, n_shifts) are skipped too
+ *   shifts         host   [n_shifts] shift amounts; n_shifts <= TESSERA_STATIC_MAX_SHIFTS, otherwise
+ *                  TESSERA_UNSUPPORTED_SHAPE and nothing is launched.  The values are copied into the
+ *                  launch itself, so the array may be freed as soon as the call returns
  * The first call on a device looks up the array's device address (once per device, with that device
  * current); make that first call before any stream capture begins.  All calls on a device share
  * the array and each call overwrites the rows it uses (nothing in it has to start at zero), so two
  * calls whose GPU work can overlap - different streams without ordering - race on it; calls on one
- * stream are safe.  Work is enqueued on `stream`; the call does not wait for it.
+ * stream are safe.  Two kernels (table fill, rotation) are enqueued on `stream`; the call does not
+ * wait for them and copies nothing from host memory.
  */
 #define TESSERA_STATIC_MAX_SHIFTS 512
-TESSERA_API int32_t tessera_rope_shift_static(const tessera_model_cfg *cfg, void *k_pool, const int32_t *slots,
-                                              const int32_t *slot_shift, int32_t n_slots, const int32_t *shifts,
-                                              int32_t n_shifts, void *stream);
+TESSERA_API int32_t tessera_rope_shift_static(const tessera_model_cfg *cfg, void *k_pool, int64_t num_pool_slots,
+                                              const int32_t *slots, const int32_t *slot_shift, int32_t n_slots,
+                                              const int32_t *shifts, int32_t n_shifts, void *stream);
 
 /*
  * Diagnostic (the paper has no counterpart): exercises the bounded wait that every kernel of this

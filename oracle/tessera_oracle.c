@@ -172,7 +172,9 @@ void oracle_rope_rotate(const double *x, double *out, int D, double delta, doubl
 /* -------------------------------------------------------------------------
  * Assembled K and V of request r (Sec. 5.3 "Preparing cache hits", "Completing
  * prefill").  For every position p < T:
- *   recomputed position j  -> K = k_new[j], V = v_new[j] (bit copies);
+ *   recomputed position j  -> K = k_new[j], V = v_new[j] (bit copies); with fresh_k_raw the fresh keys
+ *                             are un-rotated projections and K = k_new[j] rotated for position p
+ *                             (Sec. 5.3 "Completing prefill", Sec. 6.1), a bit copy only at p = 0;
  *   otherwise, cached unit u at offset i = p - target_pos(u):
  *        V = pool row (bit copy: values carry no rotation),
  *        K = pool row rotated by delta = (target_pos(u) + tstride(u) * i) - (cached_pos(u) + stride(u) * i),
@@ -182,19 +184,33 @@ void oracle_rope_rotate(const double *x, double *out, int D, double delta, doubl
  * k_asm is fp64 and left unrounded.  k_bits / k_exact: rows whose result is a bit
  * copy (recomputed rows and delta == 0) are given as bf16 bits with k_exact = 1.
  * ------------------------------------------------------------------------- */
-static uint16_t f32_to_bf16_rne(float f)
+/* Nearest bf16 (8 significant bits, float's exponent range), ties to even, of a double: ONE rounding
+ * of the exact value.  Written with frexp / nearbyint (the default rounding mode is to-nearest-even). */
+uint16_t oracle_f64_to_bf16_rne(double x)
 {
+    uint16_t sign = signbit(x) ? 0x8000 : 0;
+    double a = fabs(x), m, q;
+    int e, prec = 8;
+    float f;
     uint32_t u;
+    if (isnan(x)) return 0x7fc0;
+    if (a == 0.0) return sign;
+    if (isinf(x)) return sign | 0x7f80;
+    m = frexp(a, &e);                       /* a = m * 2^e, 0.5 <= m < 1 */
+    if (e < -125) prec = 8 - (-125 - e);    /* below 2^-126 the spacing is fixed at 2^-133 */
+    if (prec < 0) return sign;
+    q = nearbyint(ldexp(m, prec));          /* integer with at most `prec` bits (or 2^prec after a carry) */
+    a = ldexp(q, e - prec);
+    if (a >= ldexp(1.0, 128)) return sign | 0x7f80;
+    f = (float)a;                           /* exact: a has at most 8 significant bits */
     memcpy(&u, &f, sizeof u);
-    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40);   /* NaN */
-    u += 0x7fffu + ((u >> 16) & 1u);
-    return (uint16_t)(u >> 16);
+    return sign | (uint16_t)(u >> 16);
 }
 
 /* 8-bit source pools (src_fmt 1; this build's extension, see oracle_e4m3_*): a stored code c
- * stands for c * scale.  The 16-bit row that reaches the destination is the float product
- * (float)c * scale rounded to nearest-even bf16 - the precision in which the library takes that
- * decision - for V and for keys whose shift is 0; rotated keys are computed from the exact
+ * stands for c * scale.  The product of a code (4 significant bits) and a float scale (24) is exact
+ * in fp64.  The 16-bit row that reaches the destination is that exact product rounded ONCE to
+ * nearest-even bf16, for V and for keys whose shift is 0; rotated keys are computed from the exact
  * product in fp64 and left unrounded like every other rotated key. */
 int oracle_assemble_ex(int r, const int32_t *seq_len, const int32_t *unit_off,
                     const int32_t *unit_len, const int32_t *unit_cached_pos,
@@ -205,7 +221,7 @@ int oracle_assemble_ex(int r, const int32_t *seq_len, const int32_t *unit_off,
                     const void *k_pool_any, const void *v_pool_any,
                     const uint16_t *k_new, const uint16_t *v_new,
                     const int32_t *unit_src_offset /* nullable */, const int32_t *unit_target_stride /* nullable */,
-                    int src_fmt, float k_scale, float v_scale,
+                    int src_fmt, float k_scale, float v_scale, int fresh_k_raw,
                     double *k_asm, uint16_t *v_asm, uint16_t *k_bits, uint8_t *k_exact, int32_t *delta_out);
 
 int oracle_assemble(int r, const int32_t *seq_len, const int32_t *unit_off,
@@ -222,7 +238,7 @@ int oracle_assemble(int r, const int32_t *seq_len, const int32_t *unit_off,
     return oracle_assemble_ex(r, seq_len, unit_off, unit_len, unit_cached_pos, unit_cached_stride, unit_target_pos,
                               unit_page_off, unit_pages, recompute_off, recompute_pos, page_size, H_kv, D, theta,
                               inv_freq, pairing, k_pool, v_pool, k_new, v_new, unit_src_offset, unit_target_stride,
-                              0, 1.0f, 1.0f, k_asm, v_asm, k_bits, k_exact, delta_out);
+                              0, 1.0f, 1.0f, 0, k_asm, v_asm, k_bits, k_exact, delta_out);
 }
 
 int oracle_assemble_ex(int r, const int32_t *seq_len, const int32_t *unit_off,
@@ -234,7 +250,7 @@ int oracle_assemble_ex(int r, const int32_t *seq_len, const int32_t *unit_off,
                     const void *k_pool_any, const void *v_pool_any,
                     const uint16_t *k_new, const uint16_t *v_new,
                     const int32_t *unit_src_offset /* nullable */, const int32_t *unit_target_stride /* nullable */,
-                    int src_fmt, float k_scale, float v_scale,
+                    int src_fmt, float k_scale, float v_scale, int fresh_k_raw,
                     double *k_asm, uint16_t *v_asm, uint16_t *k_bits, uint8_t *k_exact, int32_t *delta_out)
 {
     const uint16_t *k_pool = (const uint16_t *)k_pool_any, *v_pool = (const uint16_t *)v_pool_any;
@@ -256,7 +272,7 @@ int oracle_assemble_ex(int r, const int32_t *seq_len, const int32_t *unit_off,
             if (src_fmt == 0) memcpy(v_asm + (size_t)p * row, v_pool + slot * row, row * sizeof(uint16_t));
             else
                 for (size_t e = 0; e < row; ++e)
-                    v_asm[(size_t)p * row + e] = f32_to_bf16_rne((float)oracle_e4m3_to_double(v_pool8[slot * row + e]) * v_scale);
+                    v_asm[(size_t)p * row + e] = oracle_f64_to_bf16_rne(oracle_e4m3_to_double(v_pool8[slot * row + e]) * (double)v_scale);
             for (int h = 0; h < H_kv; ++h) {
                 double *dst = k_asm + (size_t)p * row + (size_t)h * D;
                 for (int d = 0; d < D; ++d)
@@ -269,7 +285,7 @@ int oracle_assemble_ex(int r, const int32_t *seq_len, const int32_t *unit_off,
                 if (src_fmt == 0) memcpy(k_bits + (size_t)p * row, k_pool + slot * row, row * sizeof(uint16_t));
                 else
                     for (size_t e = 0; e < row; ++e)
-                        k_bits[(size_t)p * row + e] = f32_to_bf16_rne((float)oracle_e4m3_to_double(k_pool8[slot * row + e]) * k_scale);
+                        k_bits[(size_t)p * row + e] = oracle_f64_to_bf16_rne(oracle_e4m3_to_double(k_pool8[slot * row + e]) * (double)k_scale);
             }
             have[p] = 1;
         }
@@ -278,9 +294,20 @@ int oracle_assemble_ex(int r, const int32_t *seq_len, const int32_t *unit_off,
         int p = recompute_pos[j];
         memcpy(v_asm + (size_t)p * row, v_new + (size_t)j * row, row * sizeof(uint16_t));
         memcpy(k_bits + (size_t)p * row, k_new + (size_t)j * row, row * sizeof(uint16_t));
-        for (size_t e = 0; e < row; ++e) k_asm[(size_t)p * row + e] = bf16_to_double(k_new[(size_t)j * row + e]);
-        k_exact[p] = 1;
-        delta_out[p] = 0;
+        if (fresh_k_raw && p != 0) {
+            /* the fresh keys were handed over BEFORE rotation (Sec. 6.1: pre-RoPE keys are captured):
+             * the request's own row is the key rotated for its position p, in fp64, unrounded */
+            for (int h = 0; h < H_kv; ++h) {
+                for (int d = 0; d < D; ++d) tmp[d] = bf16_to_double(k_new[(size_t)j * row + (size_t)h * D + d]);
+                oracle_rope_rotate(tmp, k_asm + (size_t)p * row + (size_t)h * D, D, (double)p, theta, inv_freq, pairing);
+            }
+            k_exact[p] = 0;
+            delta_out[p] = p;
+        } else {
+            for (size_t e = 0; e < row; ++e) k_asm[(size_t)p * row + e] = bf16_to_double(k_new[(size_t)j * row + e]);
+            k_exact[p] = 1;
+            delta_out[p] = 0;
+        }
         have[p] = 1;
     }
     int missing = 0;

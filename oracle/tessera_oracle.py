@@ -121,6 +121,19 @@ def e4m3_decode(codes: np.ndarray) -> np.ndarray:
     return out
 
 
+def f64_to_bf16_bits(values: np.ndarray) -> np.ndarray:
+    """float64 values -> bf16 bit patterns, one round-to-nearest-even of the exact value."""
+    values = np.ascontiguousarray(values, dtype=np.float64)
+    out = np.empty(values.shape, np.uint16)
+    fn = lib().oracle_f64_to_bf16_rne
+    fn.restype = ctypes.c_uint16
+    fn.argtypes = [ctypes.c_double]
+    flat, o = values.ravel(), out.ravel()
+    for i in range(flat.size):
+        o[i] = fn(float(flat[i]))
+    return out
+
+
 def e4m3_encode(values: np.ndarray) -> np.ndarray:
     """float32 values -> uint8 e4m3 codes: nearest, ties to even, saturating at +-448."""
     values = np.ascontiguousarray(values, dtype=np.float32)
@@ -131,9 +144,10 @@ def e4m3_encode(values: np.ndarray) -> np.ndarray:
 
 def assemble(w, r: int, k_pool_bits, v_pool_bits, k_new_bits, v_new_bits,
              inv_freq: Optional[np.ndarray] = None, src_fmt: int = 0, k_scale: float = 1.0,
-             v_scale: float = 1.0) -> Assembled:
+             v_scale: float = 1.0, fresh_k_raw: bool = False) -> Assembled:
     """src_fmt 0: 16-bit source pools given as bf16 bits; 1: 8-bit (e4m3 codes, uint8) source pools,
-    a code standing for code * scale."""
+    a code standing for code * scale.  fresh_k_raw: k_new holds un-rotated keys, which the request sees
+    rotated for their positions."""
     sh = w.shape
     T = int(w.seq_len[r])
     a = Assembled(T, sh.num_kv_heads, sh.head_dim)
@@ -148,7 +162,7 @@ def assemble(w, r: int, k_pool_bits, v_pool_bits, k_new_bits, v_new_bits,
         ctypes.c_int(sh.rope_pairing),
         _p(k_pool_bits), _p(v_pool_bits), _p(k_new_bits), _p(v_new_bits),
         _p(_opt(w, "unit_src_offset")), _p(_opt(w, "unit_target_stride")),
-        ctypes.c_int(src_fmt), ctypes.c_float(k_scale), ctypes.c_float(v_scale),
+        ctypes.c_int(src_fmt), ctypes.c_float(k_scale), ctypes.c_float(v_scale), ctypes.c_int(int(fresh_k_raw)),
         _p(a.k), _p(a.v_bits), _p(a.k_bits), _p(a.k_exact), _p(a.delta))
     if st != 0:
         raise ValueError("oracle_assemble: request %d has positions nobody supplies" % r)

@@ -42,18 +42,20 @@ class ComposeDesc(ctypes.Structure):
                 ("unit_cached_pos", _I32P), ("unit_cached_stride", _I32P), ("unit_target_pos", _I32P),
                 ("unit_page_off", _I32P), ("unit_pages", _I32P), ("recompute_off", _I32P),
                 ("recompute_pos", _I32P), ("free_pages", _I32P), ("n_free", ctypes.c_int32),
-                ("unit_src_offset", _I32P), ("num_source_pages", ctypes.c_int32), ("unit_target_stride", _I32P)]
+                ("unit_src_offset", _I32P), ("num_source_pages", ctypes.c_int32), ("unit_target_stride", _I32P),
+                ("unit_retain_page_off", _I32P), ("unit_retain_pages", _I32P), ("retain_pool_pages", ctypes.c_int32)]
 
 
 class PlanInfo(ctypes.Structure):
     _fields_ = [("total_tokens", ctypes.c_int64), ("n_q", ctypes.c_int64), ("cached_tokens", ctypes.c_int64),
                 ("qk_pairs", ctypes.c_int64), ("gather_bytes", ctypes.c_int64), ("attn_flops", ctypes.c_int64),
                 ("n_rope_rows", ctypes.c_int32), ("n_gather_items", ctypes.c_int32),
-                ("n_attn_items", ctypes.c_int32), ("attn_kernel", ctypes.c_int32)]
+                ("n_attn_items", ctypes.c_int32), ("attn_kernel", ctypes.c_int32),
+                ("retained_tokens", ctypes.c_int64), ("attn_mma_pairs", ctypes.c_int64)]
 
 
 EXPORTS = ["tessera_plan_create", "tessera_plan_destroy", "tessera_plan_block_table", "tessera_plan_get_info",
-           "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_kv_compose_from_fp8", "tessera_kv_retain_fp8", "tessera_rope_shift", "tessera_rope_fresh", "tessera_partial_prefill_attn",
+           "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_kv_compose_from_fp8", "tessera_kv_retain_fp8", "tessera_rope_shift", "tessera_rope_fresh", "tessera_extend_write", "tessera_partial_prefill_attn",
            "tessera_composed_prefill_host", "tessera_rope_shift_static", "tessera_selftest_bounded_wait", "tessera_last_error",
            "tessera_launch_count"]
 
@@ -70,10 +72,11 @@ _lib.tessera_kv_compose_from_fp8.argtypes = [_vp, _vp, _vp, ctypes.c_float, ctyp
 _lib.tessera_kv_retain_fp8.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_float, ctypes.c_float, ctypes.c_uint32, _vp]
 _lib.tessera_rope_shift.argtypes = [_vp, _vp, _vp]
 _lib.tessera_rope_fresh.argtypes = [_vp, _vp, _vp, _vp]
+_lib.tessera_extend_write.argtypes = [_vp] * 9
 _lib.tessera_partial_prefill_attn.argtypes = [_vp] * 9
 _lib.tessera_composed_prefill_host.argtypes = [_vp] * 9
-_lib.tessera_rope_shift_static.argtypes = [ctypes.POINTER(ModelCfg), _vp, _vp, _vp, ctypes.c_int32, _I32P,
-                                           ctypes.c_int32, _vp]
+_lib.tessera_rope_shift_static.argtypes = [ctypes.POINTER(ModelCfg), _vp, ctypes.c_int64, _vp, _vp, ctypes.c_int32,
+                                           _I32P, ctypes.c_int32, _vp]
 _lib.tessera_selftest_bounded_wait.argtypes = [ctypes.c_int64, _I32P, ctypes.POINTER(ctypes.c_int64), _vp]
 _lib.tessera_last_error.argtypes = [ctypes.c_char_p, ctypes.c_int32]
 _lib.tessera_launch_count.argtypes = []
@@ -140,10 +143,11 @@ class Plan:
                        None if self._inv is None else self._inv.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
                        int(sh.rope_pairing), float(sh.sm_scale))
         opt = [None if getattr(w, f, None) is None else _arr(getattr(w, f))
-               for f in ("unit_src_offset", "unit_target_stride")]
+               for f in ("unit_src_offset", "unit_target_stride", "unit_retain_page_off", "unit_retain_pages")]
         op = [None if x is None else _ptr(x) for x in opt]
         desc = ComposeDesc(len(a[0]), *[_ptr(x) for x in a[:11]], len(a[10]), op[0],
-                           int(getattr(w, "num_source_pages", 0) or 0), op[1])
+                           int(getattr(w, "num_source_pages", 0) or 0), op[1], op[2], op[3],
+                           int(getattr(w, "retain_pool_pages", 0) or 0))
         self._opt = opt
         self._h = _vp()
         self.host_only = host_only
@@ -154,6 +158,9 @@ class Plan:
         self.batch = len(a[0])
         self.info = PlanInfo()
         _check(_lib.tessera_plan_get_info(self._h, ctypes.byref(self.info)))
+        # share of the tensor-core (row, key) products that is not an algorithmic (query row, key) pair
+        pairs = self.info.qk_pairs * sh.num_q_heads
+        self.masked_mma_fraction = 1.0 - pairs / self.info.attn_mma_pairs if self.info.attn_mma_pairs else 0.0
 
     def block_table(self):
         """(page_off, pages, src_slot) as numpy copies of the plan's host tables."""
@@ -200,6 +207,12 @@ class Plan:
         """Rotate fresh q / k_new rows in place for their target positions (either may be None)."""
         _check(_lib.tessera_rope_fresh(self._h, _dev(q), _dev(k_new), _stream(stream)))
 
+    def extend_write(self, k_pool, v_pool, q, k_new_raw, v_new, k_cache=None, v_cache=None, stream=None) -> None:
+        """Fused write side of the extend pass: rotate q in place, write rotated K / V rows to their slots
+        and the raw rows of captured units to k_cache / v_cache (attention then runs with k_new = v_new = None)."""
+        _check(_lib.tessera_extend_write(self._h, _dev(k_pool), _dev(v_pool), _dev(q), _dev(k_new_raw), _dev(v_new),
+                                         _dev(k_cache), _dev(v_cache), _stream(stream)))
+
     def partial_prefill_attn(self, k_pool, v_pool, q, k_new, v_new, out, lse=None, stream=None) -> None:
         _check(_lib.tessera_partial_prefill_attn(self._h, _dev(k_pool), _dev(v_pool), _dev(q), _dev(k_new),
                                                  _dev(v_new), _dev(out), _dev(lse), _stream(stream)))
@@ -233,16 +246,20 @@ def selftest_bounded_wait(max_cycles: int, stream=None):
 STATIC_MAX_SHIFTS = 512
 
 
-def rope_shift_static(shape, k_pool, slots, slot_shift, shifts, stream=None, inv_freq=None) -> None:
+def rope_shift_static(shape, k_pool, slots, slot_shift, shifts, stream=None, inv_freq=None,
+                      num_pool_slots: Optional[int] = None) -> None:
     """tessera_rope_shift_static: rotate the listed pool slots in place without any device
-    allocation.  `slots` / `slot_shift` are int32 device tensors, `shifts` a host int32 sequence."""
+    allocation.  `slots` / `slot_shift` are int32 device tensors, `shifts` a host int32 sequence;
+    `num_pool_slots` (default: every row of k_pool) bounds the slot ids the kernel accepts."""
     inv = None if inv_freq is None else np.ascontiguousarray(inv_freq, dtype=np.float64)
     cfg = ModelCfg(shape.num_q_heads, shape.num_kv_heads, shape.head_dim, shape.page_size, float(shape.rope_theta),
                    None if inv is None else inv.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
                    int(shape.rope_pairing), float(shape.sm_scale))
     sh = _arr(shifts)
-    _check(_lib.tessera_rope_shift_static(ctypes.byref(cfg), _dev(k_pool), _dev(slots), _dev(slot_shift),
-                                          int(slots.numel()), _ptr(sh), len(sh), _stream(stream)))
+    if num_pool_slots is None:
+        num_pool_slots = int(k_pool.shape[0]) * int(k_pool.shape[1])
+    _check(_lib.tessera_rope_shift_static(ctypes.byref(cfg), _dev(k_pool), int(num_pool_slots), _dev(slots),
+                                          _dev(slot_shift), int(slots.numel()), _ptr(sh), len(sh), _stream(stream)))
 
 
 def plan_create_status(w, host_only: bool = True) -> int:

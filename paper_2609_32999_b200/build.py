@@ -11,7 +11,6 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtessera.so")
 SOURCES = ["api.cu", "plan.cu", "gather_rope.cu", "kv_fp8.cu", "attn_tc.cu",
            "rope_shift_static.cu", "selftest.cu"]
-EXTRA = os.environ.get("TESSERA_NVCC_EXTRA", "").split()     # extra nvcc flags for experiments
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 
@@ -36,7 +35,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     procs = []
     for src in SOURCES:
         obj = os.path.join(CSRC, src.replace(".cu", ".o"))
-        cmd = [nvcc(), *NVCC_FLAGS, *EXTRA, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c",
+        cmd = [nvcc(), *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c",
                os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")

@@ -33,6 +33,22 @@ int32_t cuda_fail(cudaError_t e, const char *what) {
 
 size_t align_up(size_t x) { return (x + 255) & ~size_t(255); }
 
+// Multiprocessor count of the current device, asked once per device.
+int32_t device_sm_count(int *out) {
+    constexpr int kMaxDevices = 64;
+    static std::atomic<int> cache[kMaxDevices];
+    int dev = 0;
+    TS_CUDA(cudaGetDevice(&dev));
+    int n = (dev >= 0 && dev < kMaxDevices) ? cache[dev].load(std::memory_order_relaxed) : 0;
+    if (n <= 0) {
+        TS_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
+        if (n <= 0) return set_error(TESSERA_CUDA_ERROR, "device reports no multiprocessors");
+        if (dev >= 0 && dev < kMaxDevices) cache[dev].store(n, std::memory_order_relaxed);
+    }
+    *out = n;
+    return TESSERA_OK;
+}
+
 template <class T>
 size_t place(size_t &off, size_t n) {
     size_t o = off;
@@ -50,6 +66,7 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     const size_t o_items = place<GatherItem>(off, pl->items.size());
     const size_t o_rope = place<float>(off, pl->rope_table.size());
     const size_t o_fresh = place<int32_t>(off, pl->fresh_dst.size());
+    const size_t o_retain = place<int32_t>(off, pl->retain_dst.size());
     const size_t o_qpos = place<int32_t>(off, pl->recompute_pos.size());
     const size_t o_qreq = place<int32_t>(off, pl->q_req.size());
     const size_t o_poff = place<int32_t>(off, pl->page_off.size());
@@ -74,6 +91,7 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     put(o_items, pl->items.data(), pl->items.size() * sizeof(GatherItem));
     put(o_rope, pl->rope_table.data(), pl->rope_table.size() * 4);
     put(o_fresh, pl->fresh_dst.data(), pl->fresh_dst.size() * 4);
+    put(o_retain, pl->retain_dst.data(), pl->retain_dst.size() * 4);
     put(o_qpos, pl->recompute_pos.data(), pl->recompute_pos.size() * 4);
     put(o_qreq, pl->q_req.data(), pl->q_req.size() * 4);
     put(o_poff, pl->page_off.data(), pl->page_off.size() * 4);
@@ -92,6 +110,7 @@ int32_t upload(tessera_plan *pl, cudaStream_t st) {
     d.items = reinterpret_cast<GatherItem *>(db + o_items);
     d.rope = reinterpret_cast<float2 *>(db + o_rope);
     d.fresh_dst = reinterpret_cast<int32_t *>(db + o_fresh);
+    d.retain_dst = pl->retain_dst.empty() ? nullptr : reinterpret_cast<int32_t *>(db + o_retain);
     d.q_pos = reinterpret_cast<int32_t *>(db + o_qpos);
     d.q_req = reinterpret_cast<int32_t *>(db + o_qreq);
     d.page_off = reinterpret_cast<int32_t *>(db + o_poff);
@@ -165,8 +184,15 @@ int32_t tessera_plan_create(const tessera_model_cfg *cfg, const tessera_compose_
     if (!pl) return set_error(TESSERA_INVALID_ARG, "out of host memory");
     std::string err;
     int32_t st = TESSERA_INVALID_ARG;
+    int num_sms = kDefaultSMs;               // a host-only plan touches no device and is sized for a B200
+    if (!(flags & TESSERA_PLAN_HOST_ONLY)) {
+        if (int32_t rc = device_sm_count(&num_sms)) {
+            delete pl;
+            return rc;
+        }
+    }
     try {
-        st = build_plan_host(cfg, desc, num_pool_pages, pl, &err);
+        st = build_plan_host(cfg, desc, num_pool_pages, num_sms, pl, &err);
     } catch (const std::bad_alloc &) {
         err = "out of host memory while building the plan";
     }
@@ -229,6 +255,8 @@ int32_t tessera_plan_get_info(const tessera_plan *pl, tessera_plan_info *info) {
     info->n_gather_items = (int32_t)pl->items.size();
     info->n_attn_items = (int32_t)pl->work.size();
     info->attn_kernel = pl->attn_kernel;
+    info->retained_tokens = pl->retained_tokens;
+    info->attn_mma_pairs = pl->mma_pairs;
     return TESSERA_OK;
 }
 
@@ -313,6 +341,22 @@ int32_t tessera_rope_fresh(const tessera_plan *pl, void *q, void *k_new, void *s
     if (int32_t rc = check_device_plan(pl)) return rc;
     if (misaligned(q) || misaligned(k_new)) return set_error(TESSERA_INVALID_ARG, "q / k_new must be 16-byte aligned");
     TS_CUDA(launch_rope_fresh(pl, q, k_new, static_cast<cudaStream_t>(stream)));
+    return TESSERA_OK;
+}
+
+int32_t tessera_extend_write(const tessera_plan *pl, void *k_pool, void *v_pool, void *q, const void *k_new_raw,
+                             const void *v_new, void *k_cache, void *v_cache, void *stream) {
+    if (int32_t rc = check_device_plan(pl)) return rc;
+    if (!k_pool || !v_pool || misaligned(k_pool) || misaligned(v_pool))
+        return set_error(TESSERA_INVALID_ARG, "k_pool / v_pool must be non-null and 16-byte aligned");
+    if (pl->n_q > 0 && (!k_new_raw || !v_new)) return set_error(TESSERA_INVALID_ARG, "k_new_raw and v_new must be non-null");
+    if (misaligned(q) || misaligned(k_new_raw) || misaligned(v_new) || misaligned(k_cache) || misaligned(v_cache))
+        return set_error(TESSERA_INVALID_ARG, "q / k_new_raw / v_new / k_cache / v_cache must be 16-byte aligned");
+    if (pl->retained_tokens > 0 && (!k_cache || !v_cache))
+        return set_error(TESSERA_INVALID_ARG, "the plan captures units: k_cache and v_cache must be non-null");
+    if (pl->retained_tokens > 0 && pl->retain_pool_pages == 0 && (k_cache != k_pool || v_cache != v_pool))
+        return set_error(TESSERA_INVALID_ARG, "the plan's cache pages are pages of the destination pool: pass k_pool / v_pool as k_cache / v_cache");
+    TS_CUDA(launch_extend_write(pl, k_pool, v_pool, q, k_new_raw, v_new, k_cache, v_cache, static_cast<cudaStream_t>(stream)));
     return TESSERA_OK;
 }
 

@@ -683,7 +683,7 @@ cudaError_t launch_attn_tc_d(const tessera_plan *pl, void *k_pool, void *v_pool,
     const DeviceTables &d = pl->dev;
     const float scale_log2 = pl->sm_scale * 1.4426950408889634f;
     // persistent: one thread block per SM (fewer when the list is shorter)
-    const unsigned grid = (unsigned)std::min<size_t>(n_work, (size_t)kNumSMs);
+    const unsigned grid = (unsigned)std::min<size_t>(n_work, (size_t)pl->num_sms);
     attn_tc_kernel<D, kMaxPages><<<grid, kThreads, Geo<D>::kSmemAlloc, st>>>(
         tq, tk, tv, to, d.tiles, work, (int)n_work, d.q_pos, d.page_off, d.pages, d.seq_len,
         static_cast<__nv_bfloat16 *>(out), lse, Hq, g, Hkv, ps, pl->num_pool_pages, scale_log2, pl->max_parts, d.ws_o, d.ws_ml, d.status);

@@ -32,19 +32,28 @@ __device__ __forceinline__ void stg(uint4 *p, const uint4 &v) {
     asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-// Rotates 8 pairs: lo holds x_m, hi holds x_{m + D/2}, cs[i] = (cos, sin) of pair i.
-// x' = x cos - y sin, y' = y cos + x sin in fp32, one round-to-nearest-even to bf16.
+// One rotary pair in fp32: (x, y) -> (x cos - y sin, y cos + x sin).  A table entry that is exactly
+// (1, 0) - a shift of zero, or a frequency of zero - returns the inputs themselves, so such elements
+// stay bit copies (the fused multiply-add would turn -0.0 into +0.0 and 0 x Inf into NaN).
+__device__ __forceinline__ void rotate_pair(float &x, float &y, const float2 c) {
+    const bool identity = c.x == 1.f && c.y == 0.f;
+    const float a = fmaf(-y, c.y, x * c.x), b = fmaf(x, c.y, y * c.x);
+    x = identity ? x : a;
+    y = identity ? y : b;
+}
+
+// Rotates 8 pairs: lo holds x_m, hi holds x_{m + D/2}, cs[i] = (cos, sin) of pair i; one
+// round-to-nearest-even to bf16 (exact for elements that were left alone).
 __device__ __forceinline__ void rotate8(uint4 &lo, uint4 &hi, const float2 *cs) {
     uint32_t *l = reinterpret_cast<uint32_t *>(&lo);
     uint32_t *h = reinterpret_cast<uint32_t *>(&hi);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const float x0 = __uint_as_float(l[i] << 16), x1 = __uint_as_float(l[i] & 0xffff0000u);
-        const float y0 = __uint_as_float(h[i] << 16), y1 = __uint_as_float(h[i] & 0xffff0000u);
-        const float2 c0 = cs[2 * i], c1 = cs[2 * i + 1];
-        const float a0 = fmaf(-y0, c0.y, x0 * c0.x), a1 = fmaf(-y1, c1.y, x1 * c1.x);
-        const float b0 = fmaf(x0, c0.y, y0 * c0.x), b1 = fmaf(x1, c1.y, y1 * c1.x);
-        __nv_bfloat162 pa = __floats2bfloat162_rn(a0, a1), pb = __floats2bfloat162_rn(b0, b1);
+        float x0 = __uint_as_float(l[i] << 16), x1 = __uint_as_float(l[i] & 0xffff0000u);
+        float y0 = __uint_as_float(h[i] << 16), y1 = __uint_as_float(h[i] & 0xffff0000u);
+        rotate_pair(x0, y0, cs[2 * i]);
+        rotate_pair(x1, y1, cs[2 * i + 1]);
+        __nv_bfloat162 pa = __floats2bfloat162_rn(x0, x1), pb = __floats2bfloat162_rn(y0, y1);
         l[i] = *reinterpret_cast<uint32_t *>(&pa);
         h[i] = *reinterpret_cast<uint32_t *>(&pb);
     }
@@ -56,9 +65,9 @@ __device__ __forceinline__ void rotate4_interleaved(uint4 &v, const float2 *cs) 
     uint32_t *w = reinterpret_cast<uint32_t *>(&v);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const float x = __uint_as_float(w[i] << 16), y = __uint_as_float(w[i] & 0xffff0000u);
-        const float2 c = cs[i];
-        __nv_bfloat162 p = __floats2bfloat162_rn(fmaf(-y, c.y, x * c.x), fmaf(x, c.y, y * c.x));
+        float x = __uint_as_float(w[i] << 16), y = __uint_as_float(w[i] & 0xffff0000u);
+        rotate_pair(x, y, cs[i]);
+        __nv_bfloat162 p = __floats2bfloat162_rn(x, y);
         w[i] = *reinterpret_cast<uint32_t *>(&p);
     }
 }
@@ -221,26 +230,98 @@ rope_fresh_kernel(uint4 *__restrict__ q, uint4 *__restrict__ k_new, const int32_
     }
 }
 
+
+// Write side of the extend pass in one pass over the fresh rows (Sec. 5.3 "Completing prefill"; Sec. 6.1:
+// the forward path captures pre-RoPE keys and values).  A thread block owns kExtendRows consecutive
+// recompute rows: D/2 threads per row evaluate cos / sin of (position x frequency) in fp64, then the
+// block walks the rows' pair-chunk tasks.  A key task reads the un-rotated chunk pair once, stores the
+// raw bits to the captured unit's cache slot (if any), rotates and stores to the request's slot; a
+// value task copies to both; a query task rotates in place.
+constexpr int kExtendRows = 4;
+template <int D, bool INTERLEAVED>
+__global__ void __launch_bounds__(256)
+extend_write_kernel(uint4 *__restrict__ q, const uint4 *__restrict__ k_raw, const uint4 *__restrict__ v_new,
+                    uint4 *k_pool, uint4 *v_pool, uint4 *k_cache, uint4 *v_cache, const int32_t *__restrict__ q_pos, const int32_t *__restrict__ fresh_dst,
+                    const int32_t *__restrict__ retain_dst, const double *__restrict__ inv_freq, int n_q, int H_q, int H_kv) {
+    constexpr int CPH = D / 16, HALF = D / 16;
+    __shared__ float2 s_cs[kExtendRows][D / 2];
+    __shared__ int32_t s_dst[kExtendRows], s_keep[kExtendRows];
+    const int tid = threadIdx.x;
+    const int j0 = blockIdx.x * kExtendRows;
+    const int rows = min(kExtendRows, n_q - j0);
+    for (int i = tid; i < rows * (D / 2); i += 256) {
+        const int r = i / (D / 2), m = i % (D / 2);
+        double sn, cs;
+        sincos((double)q_pos[j0 + r] * inv_freq[m], &sn, &cs);
+        s_cs[r][m] = make_float2((float)cs, (float)sn);
+    }
+    if (tid < rows) {
+        s_dst[tid] = fresh_dst[j0 + tid];
+        s_keep[tid] = retain_dst ? retain_dst[j0 + tid] : -1;
+    }
+    __syncthreads();
+    const int c = tid % CPH;                        // 256 and every task count below are multiples of CPH
+    const int kv_tasks = H_kv * CPH, q_tasks = q ? H_q * CPH : 0;
+    const int row_chunks = H_kv * (D / 8);
+    // keys and values: task t of row r = head t / CPH, pair-chunk c
+    for (int t = tid; t < rows * kv_tasks; t += 256) {
+        const int r = t / kv_tasks, w = t - r * kv_tasks;
+        const int chunk = (w / CPH) * (D / 8) + c;
+        const size_t so = (size_t)(j0 + r) * row_chunks + chunk;
+        uint4 klo = ldg_stream(k_raw + so), khi = ldg_stream(k_raw + so + HALF);
+        const uint4 vlo = ldg_stream(v_new + so), vhi = ldg_stream(v_new + so + HALF);
+        const size_t dso = (size_t)s_dst[r] * row_chunks + chunk;
+        stg(v_pool + dso, vlo);
+        stg(v_pool + dso + HALF, vhi);
+        if (s_keep[r] >= 0) {
+            const size_t co = (size_t)s_keep[r] * row_chunks + chunk;
+            stg(k_cache + co, klo);
+            stg(k_cache + co + HALF, khi);
+            stg(v_cache + co, vlo);
+            stg(v_cache + co + HALF, vhi);
+        }
+        float2 cr[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cr[i] = s_cs[r][cs_index<D, INTERLEAVED>(c, i)];
+        rotate_task<INTERLEAVED>(klo, khi, cr);
+        stg(k_pool + dso, klo);
+        stg(k_pool + dso + HALF, khi);
+    }
+    // queries, in place
+    const int q_chunks = H_q * (D / 8);
+    for (int t = tid; t < rows * q_tasks; t += 256) {
+        const int r = t / q_tasks, w = t - r * q_tasks;
+        uint4 *plo = q + (size_t)(j0 + r) * q_chunks + (w / CPH) * (D / 8) + c, *phi = plo + HALF;
+        uint4 lo = ldg_plain(plo), hi = ldg_plain(phi);
+        float2 cr[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) cr[i] = s_cs[r][cs_index<D, INTERLEAVED>(c, i)];
+        rotate_task<INTERLEAVED>(lo, hi, cr);
+        stg(plo, lo);
+        stg(phi, hi);
+    }
+}
+
 template <int D, bool IL>
 cudaError_t launch_gather_d(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
-                            GatherMode mode, cudaStream_t st) {
-    const int n = (int)pl->items.size();
+                            GatherMode mode, const int32_t *g_src, int first_item, int n, cudaStream_t st) {
     if (n == 0) return cudaSuccess;
     auto *kp = static_cast<uint4 *>(k_pool);
     auto *vp = static_cast<uint4 *>(v_pool);
     auto *ks = static_cast<const uint4 *>(k_src);
     auto *vs = static_cast<const uint4 *>(v_src);
     const DeviceTables &d = pl->dev;
+    const GatherItem *items = d.items + first_item;
     const int H = pl->cfg.num_kv_heads;
     switch (mode) {
         case GatherMode::kCopy:
-            gather_rope_kernel<D, true, false, false, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            gather_rope_kernel<D, true, false, false, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, g_src, d.g_dst, items, d.rope, H);
             break;
         case GatherMode::kCopyRotate:
-            gather_rope_kernel<D, true, true, false, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            gather_rope_kernel<D, true, true, false, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, g_src, d.g_dst, items, d.rope, H);
             break;
         case GatherMode::kShiftInPlace:
-            gather_rope_kernel<D, false, true, true, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, d.g_src, d.g_dst, d.items, d.rope, H);
+            gather_rope_kernel<D, false, true, true, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, g_src, d.g_dst, items, d.rope, H);
             break;
     }
     count_launch();
@@ -249,14 +330,19 @@ cudaError_t launch_gather_d(const tessera_plan *pl, const void *k_src, const voi
 
 }  // namespace
 
-cudaError_t launch_gather(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
-                          GatherMode mode, cudaStream_t st) {
+cudaError_t launch_gather_range(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
+                                GatherMode mode, const int32_t *g_src, int first_item, int n_items, cudaStream_t st) {
     const bool il = pl->cfg.rope_pairing == 1;
     if (pl->cfg.head_dim == 128)
-        return il ? launch_gather_d<128, true>(pl, k_src, v_src, k_pool, v_pool, mode, st)
-                  : launch_gather_d<128, false>(pl, k_src, v_src, k_pool, v_pool, mode, st);
-    return il ? launch_gather_d<64, true>(pl, k_src, v_src, k_pool, v_pool, mode, st)
-              : launch_gather_d<64, false>(pl, k_src, v_src, k_pool, v_pool, mode, st);
+        return il ? launch_gather_d<128, true>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, st)
+                  : launch_gather_d<128, false>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, st);
+    return il ? launch_gather_d<64, true>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, st)
+              : launch_gather_d<64, false>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, st);
+}
+
+cudaError_t launch_gather(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
+                          GatherMode mode, cudaStream_t st) {
+    return launch_gather_range(pl, k_src, v_src, k_pool, v_pool, mode, pl->dev.g_src, 0, (int)pl->items.size(), st);
 }
 
 cudaError_t launch_rope_fresh(const tessera_plan *pl, void *q, void *k_new, cudaStream_t st) {
@@ -278,6 +364,29 @@ cudaError_t launch_rope_fresh(const tessera_plan *pl, void *q, void *k_new, cuda
     return cudaGetLastError();
 }
 
+cudaError_t launch_extend_write(const tessera_plan *pl, void *k_pool, void *v_pool, void *q, const void *k_new_raw,
+                                const void *v_new, void *k_cache, void *v_cache, cudaStream_t st) {
+    if (pl->n_q == 0) return cudaSuccess;
+    const DeviceTables &d = pl->dev;
+    const int Hq = pl->cfg.num_q_heads, Hkv = pl->cfg.num_kv_heads, n_q = (int)pl->n_q;
+    const unsigned blocks = (unsigned)((n_q + kExtendRows - 1) / kExtendRows);
+    auto *qp = static_cast<uint4 *>(q);
+    auto *kr = static_cast<const uint4 *>(k_new_raw), *vn = static_cast<const uint4 *>(v_new);
+    auto *kp = static_cast<uint4 *>(k_pool), *vp = static_cast<uint4 *>(v_pool);
+    auto *kc = static_cast<uint4 *>(k_cache), *vc = static_cast<uint4 *>(v_cache);
+    const int32_t *keep = pl->retained_tokens > 0 ? d.retain_dst : nullptr;
+    const bool il = pl->cfg.rope_pairing == 1;
+    if (pl->cfg.head_dim == 128) {
+        if (il) extend_write_kernel<128, true><<<blocks, 256, 0, st>>>(qp, kr, vn, kp, vp, kc, vc, d.q_pos, d.fresh_dst, keep, d.inv_freq, n_q, Hq, Hkv);
+        else extend_write_kernel<128, false><<<blocks, 256, 0, st>>>(qp, kr, vn, kp, vp, kc, vc, d.q_pos, d.fresh_dst, keep, d.inv_freq, n_q, Hq, Hkv);
+    } else {
+        if (il) extend_write_kernel<64, true><<<blocks, 256, 0, st>>>(qp, kr, vn, kp, vp, kc, vc, d.q_pos, d.fresh_dst, keep, d.inv_freq, n_q, Hq, Hkv);
+        else extend_write_kernel<64, false><<<blocks, 256, 0, st>>>(qp, kr, vn, kp, vp, kc, vc, d.q_pos, d.fresh_dst, keep, d.inv_freq, n_q, Hq, Hkv);
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_pool, const void *k_new,
                                  const void *v_new, int chunk, cudaStream_t st) {
     if (pl->n_q == 0 || (!k_new && !v_new)) return cudaSuccess;
@@ -286,7 +395,7 @@ cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_p
     const int64_t rows = chunk < 0 ? pl->n_q : pl->chunk_row_off[chunk + 1] - row0;
     if (rows == 0) return cudaSuccess;
     const int64_t n_chunks = rows * row_chunks;
-    const int blocks = (int)std::min<int64_t>((n_chunks + 255) / 256, 148 * 16);
+    const int blocks = (int)std::min<int64_t>((n_chunks + 255) / 256, (int64_t)pl->num_sms * 16);
     scatter_fresh_kernel<<<blocks, 256, 0, st>>>(static_cast<uint4 *>(k_pool), static_cast<uint4 *>(v_pool),
                                                 static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new),
                                                 pl->dev.fresh_dst, row0 * row_chunks, n_chunks, row_chunks);

@@ -65,26 +65,26 @@ __device__ __forceinline__ uint2 pack_e4m3x8(const float (&f)[8], float mul) {
     return make_uint2(w[0], w[1]);
 }
 
-// x' = x cos - y sin, y' = y cos + x sin in fp32, the arithmetic of the 16-bit gather.
+// x' = x cos - y sin, y' = y cos + x sin in fp32, the arithmetic of the 16-bit gather; a table entry
+// that is exactly (1, 0) leaves the pair untouched (signed zeros and infinities survive a zero shift).
+__device__ __forceinline__ void rotate_pair(float &x, float &y, const float2 c) {
+    const bool identity = c.x == 1.f && c.y == 0.f;
+    const float a = fmaf(-y, c.y, x * c.x), b = fmaf(x, c.y, y * c.x);
+    x = identity ? x : a;
+    y = identity ? y : b;
+}
 template <bool INTERLEAVED>
 __device__ __forceinline__ void rotate_f(float (&lo)[8], float (&hi)[8], const float2 *cs) {
     if (INTERLEAVED) {
         // lo holds pairs (0,1) (2,3) .. with cs[0..3]; hi the chunk D/2 elements later with cs[4..7]
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float x = lo[2 * i], y = lo[2 * i + 1], u = hi[2 * i], v = hi[2 * i + 1];
-            lo[2 * i] = fmaf(-y, cs[i].y, x * cs[i].x);
-            lo[2 * i + 1] = fmaf(x, cs[i].y, y * cs[i].x);
-            hi[2 * i] = fmaf(-v, cs[4 + i].y, u * cs[4 + i].x);
-            hi[2 * i + 1] = fmaf(u, cs[4 + i].y, v * cs[4 + i].x);
+            rotate_pair(lo[2 * i], lo[2 * i + 1], cs[i]);
+            rotate_pair(hi[2 * i], hi[2 * i + 1], cs[4 + i]);
         }
     } else {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float x = lo[i], y = hi[i];
-            lo[i] = fmaf(-y, cs[i].y, x * cs[i].x);
-            hi[i] = fmaf(x, cs[i].y, y * cs[i].x);
-        }
+        for (int i = 0; i < 8; ++i) rotate_pair(lo[i], hi[i], cs[i]);
     }
 }
 template <int D, bool INTERLEAVED>
@@ -184,36 +184,43 @@ kv_fp8_kernel(const void *__restrict__ k_src, const void *__restrict__ v_src, vo
 
 template <int D, bool TO_8BIT, bool IL>
 cudaError_t launch_d(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst, bool rotate,
-                     float k_mul, float v_mul, cudaStream_t st) {
-    const int n = (int)pl->items.size();
+                     float k_mul, float v_mul, const int32_t *g_src, int first_item, int n, cudaStream_t st) {
     if (n == 0) return cudaSuccess;
     const DeviceTables &d = pl->dev;
+    const GatherItem *items = d.items + first_item;
     const int H = pl->cfg.num_kv_heads;
     if (rotate)
-        kv_fp8_kernel<D, TO_8BIT, true, IL><<<n, kThreads, 0, st>>>(k_src, v_src, k_dst, v_dst, d.g_src, d.g_dst, d.items, d.rope, H, k_mul, v_mul);
+        kv_fp8_kernel<D, TO_8BIT, true, IL><<<n, kThreads, 0, st>>>(k_src, v_src, k_dst, v_dst, g_src, d.g_dst, items, d.rope, H, k_mul, v_mul);
     else
-        kv_fp8_kernel<D, TO_8BIT, false, IL><<<n, kThreads, 0, st>>>(k_src, v_src, k_dst, v_dst, d.g_src, d.g_dst, d.items, d.rope, H, k_mul, v_mul);
+        kv_fp8_kernel<D, TO_8BIT, false, IL><<<n, kThreads, 0, st>>>(k_src, v_src, k_dst, v_dst, g_src, d.g_dst, items, d.rope, H, k_mul, v_mul);
     count_launch();
     return cudaGetLastError();
 }
 
 template <bool TO_8BIT>
 cudaError_t launch_dir(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst, bool rotate,
-                       float k_mul, float v_mul, cudaStream_t st) {
+                       float k_mul, float v_mul, const int32_t *g_src, int first_item, int n, cudaStream_t st) {
     const bool il = pl->cfg.rope_pairing == 1;
     if (pl->cfg.head_dim == 128)
-        return il ? launch_d<128, TO_8BIT, true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st)
-                  : launch_d<128, TO_8BIT, false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st);
-    return il ? launch_d<64, TO_8BIT, true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st)
-              : launch_d<64, TO_8BIT, false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st);
+        return il ? launch_d<128, TO_8BIT, true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, st)
+                  : launch_d<128, TO_8BIT, false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, st);
+    return il ? launch_d<64, TO_8BIT, true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, st)
+              : launch_d<64, TO_8BIT, false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, st);
 }
 
 }  // namespace
 
+cudaError_t launch_kv_fp8_range(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst,
+                                bool to_8bit, bool rotate, float k_mul, float v_mul, const int32_t *g_src, int first_item,
+                                int n_items, cudaStream_t st) {
+    return to_8bit ? launch_dir<true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n_items, st)
+                   : launch_dir<false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n_items, st);
+}
+
 cudaError_t launch_kv_fp8(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst,
                           bool to_8bit, bool rotate, float k_mul, float v_mul, cudaStream_t st) {
-    return to_8bit ? launch_dir<true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st)
-                   : launch_dir<false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, st);
+    return launch_kv_fp8_range(pl, k_src, v_src, k_dst, v_dst, to_8bit, rotate, k_mul, v_mul, pl->dev.g_src, 0,
+                               (int)pl->items.size(), st);
 }
 
 }  // namespace tessera

@@ -14,12 +14,23 @@ void count_launch();   // bumps the process-wide kernel-launch counter
 // separate source pool - and written to the plan's destination slots in (k_pool, v_pool).
 cudaError_t launch_gather(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
                           GatherMode mode, cudaStream_t st);
+// The same kernel over items [first_item, first_item + n_items) of the plan, with the source slots taken
+// from `g_src` (device, indexed like the plan's copy list) instead of the plan's own list.
+cudaError_t launch_gather_range(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
+                                GatherMode mode, const int32_t *g_src, int first_item, int n_items, cudaStream_t st);
+cudaError_t launch_kv_fp8_range(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst,
+                                bool to_8bit, bool rotate, float k_mul, float v_mul, const int32_t *g_src, int first_item,
+                                int n_items, cudaStream_t st);
 // 8-bit (e4m3) tier.  to_8bit false: (k_src, v_src) hold codes, (k_dst, v_dst) 16-bit pages, mul = scale;
 // to_8bit true: the reverse, mul = 1 / scale.  Copy list and shift table are the plan's.
 cudaError_t launch_kv_fp8(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst,
                           bool to_8bit, bool rotate, float k_mul, float v_mul, cudaStream_t st);
 // In-place rotation of the fresh q / k_new rows for their target positions (either may be null).
 cudaError_t launch_rope_fresh(const tessera_plan *pl, void *q, void *k_new, cudaStream_t st);
+// Fused write side of the extend pass: rotate q in place, write rotated K / V rows to their slots and raw
+// K / V rows of captured units to their cache slots (k_cache / v_cache may be null when nothing is captured).
+cudaError_t launch_extend_write(const tessera_plan *pl, void *k_pool, void *v_pool, void *q, const void *k_new_raw,
+                                const void *v_new, void *k_cache, void *v_cache, cudaStream_t st);
 // chunk < 0: the whole batch; otherwise only request chunk `chunk` (see tessera_plan::chunk_row_off).
 // k_new / v_new / q / out / lse always point at row 0 of the whole batch.
 cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_pool, const void *k_new,

@@ -26,9 +26,11 @@ bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 }  // namespace
 
 int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc *d,
-                        int32_t num_pool_pages, tessera_plan *pl, std::string *err) {
+                        int32_t num_pool_pages, int num_sms, tessera_plan *pl, std::string *err) {
     auto fail = [&](int32_t code, const std::string &msg) { *err = msg; return code; };
     if (!cfg || !d || !pl) return fail(TESSERA_INVALID_ARG, "null cfg / desc / plan");
+    if (num_sms <= 0) return fail(TESSERA_INVALID_ARG, "multiprocessor count must be positive");
+    pl->num_sms = num_sms;
     if (d->batch < 0 || num_pool_pages < 0 || d->n_free < 0)
         return fail(TESSERA_INVALID_ARG, "negative batch, pool size or free-list length");
     if (d->batch > 0 && (!d->seq_len || !d->unit_off || !d->recompute_off))
@@ -91,7 +93,20 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
                 return fail(TESSERA_INVALID_ARG, fmt("unit %ld: cached stride must be 0 or 1", u));
         }
         if (d->unit_page_off[n_units] > 0 && !d->unit_pages) return fail(TESSERA_INVALID_ARG, "null unit_pages");
+        if (d->unit_retain_page_off) {
+            if (d->unit_retain_page_off[0] != 0) return fail(TESSERA_INVALID_ARG, "unit_retain_page_off must start at 0");
+            for (int u = 0; u < n_units; ++u) {
+                const int np = d->unit_retain_page_off[u + 1] - d->unit_retain_page_off[u];
+                if (np < 0) return fail(TESSERA_INVALID_ARG, fmt("unit %ld: unit_retain_page_off decreases", u));
+                if (np != 0 && np != (d->unit_len[u] + B - 1) / B)
+                    return fail(TESSERA_INVALID_ARG, fmt("unit %ld: %ld cache pages for %ld tokens", u, np, d->unit_len[u]));
+            }
+            if (d->unit_retain_page_off[n_units] > 0 && !d->unit_retain_pages) return fail(TESSERA_INVALID_ARG, "null unit_retain_pages");
+        }
     }
+    if (d->retain_pool_pages < 0) return fail(TESSERA_INVALID_ARG, "negative retain_pool_pages");
+    if ((int64_t)d->retain_pool_pages * B > (int64_t)INT32_MAX) return fail(TESSERA_UNSUPPORTED_SHAPE, "cache pool has more than 2^31 slots");
+    pl->retain_pool_pages = d->retain_pool_pages;
 
     // ---- block tables: request r takes the next ceil(T_r / B) free pages
     pl->seq_len.assign(d->seq_len, d->seq_len + batch);
@@ -127,6 +142,22 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
         page_use[pg] = 2;
     }
 
+    // cache pages of captured units: in range, distinct, and - when they live in the destination pool -
+    // neither sources nor destinations of this batch
+    const int n_retain_pages = (n_units && d->unit_retain_page_off) ? d->unit_retain_page_off[n_units] : 0;
+    if (n_retain_pages > 0) {
+        const int limit = d->retain_pool_pages > 0 ? d->retain_pool_pages : num_pool_pages;
+        std::vector<uint8_t> seen(limit, 0);
+        for (int k = 0; k < n_retain_pages; ++k) {
+            const int pg = d->unit_retain_pages[k];
+            if (pg < 0 || pg >= limit) return fail(TESSERA_PAGE_OUT_OF_RANGE, fmt("cache page %ld outside pool of %ld pages", pg, limit));
+            if (seen[pg]) return fail(TESSERA_PAGE_OUT_OF_RANGE, fmt("cache page %ld listed twice", pg));
+            seen[pg] = 1;
+            if (d->retain_pool_pages == 0 && page_use[pg] != 0)
+                return fail(TESSERA_PAGE_OUT_OF_RANGE, fmt("cache page %ld is also a source or destination page of this batch", pg));
+        }
+    }
+
     // ---- per-position sources, recompute rows, coverage
     pl->src_slot.assign((size_t)total, -1);
     pl->recompute_off.assign(d->recompute_off, d->recompute_off + batch + 1);
@@ -136,6 +167,9 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
     pl->g_src.clear(); pl->g_dst.clear(); pl->items.clear();
     std::vector<int32_t> unit_of((size_t)total, -1);
     std::vector<uint8_t> fresh((size_t)total, 0);
+    std::vector<int32_t> fresh_row((size_t)total, -1);     // recompute row index of a position
+    pl->retain_dst.assign(n_retain_pages > 0 ? n_q : 0, -1);
+    pl->retained_tokens = 0;
     std::vector<int64_t> deltas;     // shift amounts needed, with repeats
     pl->qk_pairs = 0;
     for (int r = 0; r < batch; ++r) {
@@ -162,6 +196,7 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
             if (j > d->recompute_off[r] && d->recompute_pos[j - 1] >= p)
                 return fail(TESSERA_UNSORTED_POSITIONS, fmt("request %ld: recompute positions not strictly ascending at index %ld", r, j));
             fresh[base + p] = 1;
+            fresh_row[base + p] = j;
             pl->q_req[j] = r;
             pl->fresh_dst[j] = pl->pages[pl->page_off[r] + p / B] * B + p % B;
             pl->qk_pairs += (int64_t)p + 1;
@@ -169,6 +204,19 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
         for (int p = 0; p < T; ++p)
             if (pl->src_slot[base + p] < 0 && !fresh[base + p])
                 return fail(TESSERA_UNCOVERED_POSITION, fmt("request %ld: position %ld has no cached unit and is not recomputed", r, p));
+        // captured units: every token is a recompute row; row j also goes to the unit's cache slot
+        if (n_retain_pages > 0)
+            for (int u = d->unit_off[r]; u < d->unit_off[r + 1]; ++u) {
+                const int first = d->unit_retain_page_off[u], np = d->unit_retain_page_off[u + 1] - first;
+                if (np == 0) continue;
+                for (int i = 0; i < d->unit_len[u]; ++i) {
+                    const int j = fresh_row[base + d->unit_target_pos[u] + i];
+                    if (j < 0)
+                        return fail(TESSERA_INVALID_ARG, fmt("unit %ld is to be captured but its token %ld is not recomputed", u, i));
+                    pl->retain_dst[j] = d->unit_retain_pages[first + i / B] * B + i % B;
+                }
+                pl->retained_tokens += d->unit_len[u];
+            }
     }
 
     // ---- copy list + shift table.  One item = up to kGatherItemTokens rows of one unit.
@@ -203,7 +251,7 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
         int64_t cached = 0;
         for (int u = 0; u < n_units; ++u)
             if (d->unit_page_off[u + 1] > d->unit_page_off[u]) cached += d->unit_len[u];
-        while (item_tokens > 8 && cached / item_tokens < 4 * 148) item_tokens /= 2;
+        while (item_tokens > 8 && cached / item_tokens < 4 * num_sms) item_tokens /= 2;
     }
     pl->cached_tokens = 0;
     for (int r = 0; r < batch; ++r)
@@ -259,10 +307,10 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
         // Split-KV: a batch with fewer items than SMs (a single request, typically) splits each item's
         // key range into parts that run as separate thread blocks and are merged afterwards.
         pl->max_parts = 1;
-        if (!pairs.empty() && (int)pairs.size() * Hkv < kSplitTargetBlocks) {
+        if (!pairs.empty() && (int)pairs.size() * Hkv < num_sms) {
             int longest = 1;
             for (auto &pr : pairs) longest = std::max(longest, steps_of(pr.second >= 0 ? pr.second : pr.first));
-            const int want = kSplitTargetBlocks / ((int)pairs.size() * Hkv);     // stay within one wave of blocks
+            const int want = num_sms / ((int)pairs.size() * Hkv);     // stay within one wave of blocks
             pl->max_parts = std::max(1, std::min({want, kSplitMaxParts, longest / kSplitMinSteps}));
         }
         pl->combine.clear();
@@ -297,6 +345,8 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
             if (w.tile_b >= 0) c += std::min(w.step_end, steps_of(w.tile_b)) - w.step_begin;
             w.cost = c;
         }
+        pl->mma_pairs = 0;
+        for (const AttnWork &w : pl->work) pl->mma_pairs += (int64_t)w.cost * kAttnTileRows * page;
         auto cost = [](const AttnWork &w) { return w.cost; };
         auto sort_items = [&](std::vector<AttnWork>::iterator first_it, std::vector<AttnWork>::iterator last_it) {
             int max_cost = 1;

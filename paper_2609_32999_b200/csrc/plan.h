@@ -13,8 +13,7 @@ namespace tessera {
 
 constexpr int kGatherItemTokens = 32;   // token rows per thread block of the gather kernel
 constexpr int kAttnTileRows = 128;      // query rows (tokens x grouped heads) per tcgen05 tile
-constexpr int kNumSMs = 148;              // thread blocks of the persistent attention kernel: one per SM of a B200
-constexpr int kSplitTargetBlocks = 148;  // split-KV aims at about this many thread blocks when a batch has fewer items
+constexpr int kDefaultSMs = 148;         // SM count assumed by a host-only plan (a B200); device plans ask the device
 constexpr int kSplitMinSteps = 4;        // never split below this many 128-key steps per part
 constexpr int kSplitMaxParts = 8;
 constexpr int kHostChunks = 4;          // request chunks of the host-buffer entry point's copy / compute pipeline
@@ -52,6 +51,7 @@ struct DeviceTables {
     GatherItem *items = nullptr;
     float2 *rope = nullptr;        // [n_rope_rows][D/2] (cos, sin)
     int32_t *fresh_dst = nullptr;  // [n_q] destination slot of each recompute row
+    int32_t *retain_dst = nullptr; // [n_q] cache slot of a captured row, -1 otherwise (null: nothing is captured)
     int32_t *q_pos = nullptr;      // [n_q]
     int32_t *q_req = nullptr;      // [n_q]
     int32_t *page_off = nullptr;   // [batch+1]
@@ -81,9 +81,14 @@ struct tessera_plan {
     int32_t batch = 0;
     bool host_only = false;
     int device = -1;
+    int num_sms = tessera::kDefaultSMs;    // multiprocessors of the plan's device: grid of the persistent attention
+                                           // kernel, target block count of split-KV and of the small-batch gather
 
     std::vector<int32_t> seq_len, tok_off, page_off, pages, src_slot;
     std::vector<int32_t> recompute_off, recompute_pos, q_req, fresh_dst;
+    std::vector<int32_t> retain_dst;       // [n_q] or empty: cache slot of every captured recompute row
+    int32_t retain_pool_pages = 0;         // > 0: captured units go to a separate cache pool of this many pages
+    int64_t retained_tokens = 0;
     std::vector<int32_t> g_src, g_dst;
     std::vector<tessera::GatherItem> items;
     std::vector<int32_t> rope_delta;       // sorted distinct shift amounts
@@ -99,7 +104,7 @@ struct tessera_plan {
     int32_t attn_kernel = 0;
     int32_t tile_tokens = 0;
 
-    int64_t total_tokens = 0, n_q = 0, cached_tokens = 0, qk_pairs = 0;
+    int64_t total_tokens = 0, n_q = 0, cached_tokens = 0, qk_pairs = 0, mma_pairs = 0;
 
     std::vector<char> host_blob;           // staging image of the device tables
     tessera::DeviceTables dev;
@@ -111,6 +116,7 @@ struct tessera_plan {
 
 namespace tessera {
 // Builds and validates all host tables.  Returns a status; on failure `err` holds the reason.
+// `num_sms`: multiprocessor count the work lists are sized for.
 int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc *desc,
-                        int32_t num_pool_pages, tessera_plan *plan, std::string *err);
+                        int32_t num_pool_pages, int num_sms, tessera_plan *plan, std::string *err);
 }  // namespace tessera

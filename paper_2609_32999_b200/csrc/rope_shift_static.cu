@@ -8,7 +8,6 @@
 #include <cmath>
 #include <cstring>
 #include <string>
-#include <vector>
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -32,19 +31,48 @@ static __device__ __align__(256) float2 g_rope_scratch[kMaxShifts * kMaxHalf];
 constexpr int kMaxDevices = 64;
 float2 *g_scratch_addr[kMaxDevices] = {};               // device address of the array, per device
 
+// The call's shift amounts and rotary frequencies travel by value as a kernel parameter (2.5 KB), so
+// no host buffer has to outlive the call and nothing is copied from pageable memory.
+struct ShiftParams {
+    int32_t shifts[kMaxShifts];
+    double inv_freq[kMaxHalf];
+};
+
+// Fills rows [0, n_shifts) of the scratch table: one thread block per shift amount, thread m
+// evaluates the angle shift x frequency_m, its cosine and sine in fp64 and stores them as fp32.
+__global__ void __launch_bounds__(kMaxHalf)
+rope_static_fill_kernel(const __grid_constant__ ShiftParams prm, float2 *__restrict__ table, int half) {
+    const int m = threadIdx.x;
+    if (m >= half) return;
+    double sn, cs;
+    sincos((double)prm.shifts[blockIdx.x] * prm.inv_freq[m], &sn, &cs);
+    table[(size_t)blockIdx.x * half + m] = make_float2((float)cs, (float)sn);
+}
+
+// (x, y) -> (x cos - y sin, y cos + x sin) in fp32; an entry that is exactly (1, 0) leaves the pair's
+// bits alone, so a zero shift is a bit copy (signed zeros included).
+__device__ __forceinline__ void rotate_pair(float &x, float &y, const float2 c) {
+    const bool identity = c.x == 1.f && c.y == 0.f;
+    const float a = fmaf(-y, c.y, x * c.x), b = fmaf(x, c.y, y * c.x);
+    x = identity ? x : a;
+    y = identity ? y : b;
+}
+
 // One warp per slot: lane handles pair-chunks (a 16-byte chunk of a head's first half and its
-// partner D/2 elements later), exactly the arithmetic of the plan-based shift kernel.
+// partner D/2 elements later), the arithmetic of the plan-based shift kernel.  A listed slot outside
+// [0, num_pool_slots) or a shift index outside the table is skipped, never dereferenced.
 template <int D>
 __global__ void __launch_bounds__(256)
 rope_shift_static_kernel(uint4 *__restrict__ k_pool, const int32_t *__restrict__ slots,
-                         const int32_t *__restrict__ slot_shift, int n, int n_shifts,
+                         const int32_t *__restrict__ slot_shift, int n, int n_shifts, int64_t num_pool_slots,
                          const float2 *__restrict__ table, int H_kv) {
     constexpr int CPH = D / 16, HALF = D / 16;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (warp >= n) return;
     const int row = slot_shift[warp];
-    if (row < 0 || row >= n_shifts) return;             // never index outside the table
-    const size_t base = (size_t)slots[warp] * (H_kv * (D / 8));
+    const int64_t slot = slots[warp];
+    if (row < 0 || row >= n_shifts || slot < 0 || slot >= num_pool_slots) return;
+    const size_t base = (size_t)slot * (H_kv * (D / 8));
     const float2 *cs = table + (size_t)row * (D / 2);
     for (int t = lane; t < H_kv * CPH; t += 32) {
         const int c = t % CPH;
@@ -53,11 +81,11 @@ rope_shift_static_kernel(uint4 *__restrict__ k_pool, const int32_t *__restrict__
         uint32_t *l = reinterpret_cast<uint32_t *>(&lo), *h = reinterpret_cast<uint32_t *>(&hi);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const float x0 = __uint_as_float(l[i] << 16), x1 = __uint_as_float(l[i] & 0xffff0000u);
-            const float y0 = __uint_as_float(h[i] << 16), y1 = __uint_as_float(h[i] & 0xffff0000u);
-            const float2 c0 = cs[c * 8 + 2 * i], c1 = cs[c * 8 + 2 * i + 1];
-            __nv_bfloat162 pa = __floats2bfloat162_rn(fmaf(-y0, c0.y, x0 * c0.x), fmaf(-y1, c1.y, x1 * c1.x));
-            __nv_bfloat162 pb = __floats2bfloat162_rn(fmaf(x0, c0.y, y0 * c0.x), fmaf(x1, c1.y, y1 * c1.x));
+            float x0 = __uint_as_float(l[i] << 16), x1 = __uint_as_float(l[i] & 0xffff0000u);
+            float y0 = __uint_as_float(h[i] << 16), y1 = __uint_as_float(h[i] & 0xffff0000u);
+            rotate_pair(x0, y0, cs[c * 8 + 2 * i]);
+            rotate_pair(x1, y1, cs[c * 8 + 2 * i + 1]);
+            __nv_bfloat162 pa = __floats2bfloat162_rn(x0, x1), pb = __floats2bfloat162_rn(y0, y1);
             l[i] = *reinterpret_cast<uint32_t *>(&pa);
             h[i] = *reinterpret_cast<uint32_t *>(&pb);
         }
@@ -68,11 +96,12 @@ rope_shift_static_kernel(uint4 *__restrict__ k_pool, const int32_t *__restrict__
 
 }  // namespace
 
-extern "C" int32_t tessera_rope_shift_static(const tessera_model_cfg *cfg, void *k_pool, const int32_t *slots,
-                                             const int32_t *slot_shift, int32_t n_slots, const int32_t *shifts,
-                                             int32_t n_shifts, void *stream) {
+extern "C" int32_t tessera_rope_shift_static(const tessera_model_cfg *cfg, void *k_pool, int64_t num_pool_slots,
+                                             const int32_t *slots, const int32_t *slot_shift, int32_t n_slots,
+                                             const int32_t *shifts, int32_t n_shifts, void *stream) {
     using tessera::api_set_error;
-    if (!cfg || !k_pool || n_slots < 0 || n_shifts < 0 || (n_slots > 0 && (!slots || !slot_shift || !shifts)))
+    if (!cfg || !k_pool || n_slots < 0 || n_shifts < 0 || num_pool_slots < 0 ||
+        (n_slots > 0 && (!slots || !slot_shift || !shifts)))
         return api_set_error(TESSERA_INVALID_ARG, "rope_shift_static: null pointer or negative count");
     if ((reinterpret_cast<uintptr_t>(k_pool) & 15) != 0)
         return api_set_error(TESSERA_INVALID_ARG, "rope_shift_static: k_pool must be 16-byte aligned");
@@ -92,7 +121,7 @@ extern "C" int32_t tessera_rope_shift_static(const tessera_model_cfg *cfg, void 
     if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices)
         return api_set_error(TESSERA_CUDA_ERROR, std::string("rope_shift_static: cudaGetDevice: ") + cudaGetErrorString(e));
     if (!g_scratch_addr[dev]) {
-        // The array's name is only a host-side handle; the kernel needs its address on THIS device.
+        // The array's name is only a host-side handle; the kernels need its address on THIS device.
         float2 *p = nullptr;
         e = cudaGetSymbolAddress(reinterpret_cast<void **>(&p), g_rope_scratch);
         if (e != cudaSuccess || !p)
@@ -101,25 +130,21 @@ extern "C" int32_t tessera_rope_shift_static(const tessera_model_cfg *cfg, void 
     }
     float2 *table = g_scratch_addr[dev];
 
-    // cos/sin in fp64, one rounding to fp32 - the same numbers the plan-based path tabulates.
-    std::vector<float> host_table((size_t)n_shifts * (D / 2) * 2);   // host memory only; staged by the copy below
-    for (int r = 0; r < n_shifts; ++r)
-        for (int m = 0; m < D / 2; ++m) {
-            const double w = cfg->inv_freq ? cfg->inv_freq[m] : std::pow(cfg->rope_theta, -2.0 * m / D);
-            const double ang = (double)shifts[r] * w;
-            host_table[(r * (D / 2) + m) * 2 + 0] = (float)std::cos(ang);
-            host_table[(r * (D / 2) + m) * 2 + 1] = (float)std::sin(ang);
-        }
+    // Frequencies are fixed on the host (the numbers the plan-based path uses); the angles, cosines
+    // and sines are evaluated by the fill kernel in fp64 and rounded once to fp32.
+    static thread_local ShiftParams prm;
+    std::memcpy(prm.shifts, shifts, sizeof(int32_t) * (size_t)n_shifts);
+    for (int m = 0; m < D / 2; ++m)
+        prm.inv_freq[m] = cfg->inv_freq ? cfg->inv_freq[m] : std::pow(cfg->rope_theta, -2.0 * m / D);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    e = cudaMemcpyAsync(table, host_table.data(), (size_t)n_shifts * (D / 2) * sizeof(float2), cudaMemcpyHostToDevice, st);
-    if (e != cudaSuccess)
-        return api_set_error(TESSERA_CUDA_ERROR, std::string("rope_shift_static: table upload: ") + cudaGetErrorString(e));
+    rope_static_fill_kernel<<<n_shifts, kMaxHalf, 0, st>>>(prm, table, D / 2);
+    tessera::count_launch();
     const int blocks = (n_slots + 7) / 8;
     auto *kp = static_cast<uint4 *>(k_pool);
     if (D == 128)
-        rope_shift_static_kernel<128><<<blocks, 256, 0, st>>>(kp, slots, slot_shift, n_slots, n_shifts, table, H);
+        rope_shift_static_kernel<128><<<blocks, 256, 0, st>>>(kp, slots, slot_shift, n_slots, n_shifts, num_pool_slots, table, H);
     else
-        rope_shift_static_kernel<64><<<blocks, 256, 0, st>>>(kp, slots, slot_shift, n_slots, n_shifts, table, H);
+        rope_shift_static_kernel<64><<<blocks, 256, 0, st>>>(kp, slots, slot_shift, n_slots, n_shifts, num_pool_slots, table, H);
     tessera::count_launch();
     e = cudaGetLastError();
     if (e != cudaSuccess)

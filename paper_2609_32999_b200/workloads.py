@@ -55,6 +55,9 @@ class Workload:
     unit_src_offset: Optional[np.ndarray] = None     # [n_units] token 0's offset inside its first source page
     unit_target_stride: Optional[np.ndarray] = None  # [n_units] 0 = every token rotated for target_pos
     num_source_pages: int = 0                        # > 0: unit_pages index a separate source pool (host tier)
+    unit_retain_page_off: Optional[np.ndarray] = None  # [n_units+1] CSR: cache pages of units captured by extend_write
+    unit_retain_pages: Optional[np.ndarray] = None
+    retain_pool_pages: int = 0                       # > 0: the cache pages index a separate cache pool
 
     @property
     def batch(self) -> int:

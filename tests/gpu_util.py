@@ -84,7 +84,8 @@ def check_assembled(g, requests=None, scattered=True):
     errs = []
     for r in (range(w.batch) if requests is None else requests):
         a = orc.assemble(w, r, g.k_before, g.v_before, g.kn_bits, g.vn_bits, src_fmt=getattr(g, "src_fmt", 0),
-                         k_scale=getattr(g, "k_scale", 1.0), v_scale=getattr(g, "v_scale", 1.0))
+                         k_scale=getattr(g, "k_scale", 1.0), v_scale=getattr(g, "v_scale", 1.0),
+                         fresh_k_raw=getattr(g, "fresh_k_raw", False))
         asm[r] = a
         T = int(w.seq_len[r])
         if T == 0:
@@ -98,9 +99,20 @@ def check_assembled(g, requests=None, scattered=True):
             keep &= g.src_slot[tok0:tok0 + T] >= 0
         else:
             keep = np.ones(T, bool)
-        assert np.array_equal(gv[keep], a.v_bits.reshape(T, row)[keep]), "V rows must be bit copies (request %d)" % r
         ex = (a.k_exact != 0) & keep
-        assert np.array_equal(gk[ex], a.k_bits.reshape(T, row)[ex]), "exact K rows differ (request %d)" % r
+        if getattr(g, "src_fmt", 0) == 1:
+            # 8-bit sources: the oracle rounds the exact product code * scale once; the library rounds
+            # the fp32 product.  The two agree bit for bit when the scale is a power of two (the product
+            # is then exact in fp32); otherwise they may differ by one bf16 step at a double-rounding tie.
+            cached_rows = keep & (g.src_slot[int(np.sum(w.seq_len[:r])):int(np.sum(w.seq_len[:r])) + T] >= 0)
+            fresh_rows = keep & ~cached_rows
+            assert np.array_equal(gv[fresh_rows], a.v_bits.reshape(T, row)[fresh_rows])
+            _expanded_rows_equal(g, gv[cached_rows], a.v_bits.reshape(T, row)[cached_rows], g.v_scale, "V (request %d)" % r)
+            _expanded_rows_equal(g, gk[ex & cached_rows], a.k_bits.reshape(T, row)[ex & cached_rows], g.k_scale, "K (request %d)" % r)
+            assert np.array_equal(gk[ex & fresh_rows], a.k_bits.reshape(T, row)[ex & fresh_rows])
+        else:
+            assert np.array_equal(gv[keep], a.v_bits.reshape(T, row)[keep]), "V rows must be bit copies (request %d)" % r
+            assert np.array_equal(gk[ex], a.k_bits.reshape(T, row)[ex]), "exact K rows differ (request %d)" % r
         rot = (a.k_exact == 0) & keep
         if rot.any():
             d = np.abs(orc.bf16_bits_to_f64(gk[rot]) - a.k.reshape(T, row)[rot])
@@ -113,6 +125,30 @@ def check_assembled(g, requests=None, scattered=True):
     else:
         mx = mean = 0.0
     return asm, mx, mean
+
+
+def _is_pow2(x: float) -> bool:
+    m, _ = np.frexp(np.float32(x))
+    return float(m) == 0.5
+
+
+def _expanded_rows_equal(g, got, want, scale, what):
+    """Rows expanded from 8-bit codes: bit-exact for a power-of-two scale; otherwise any difference must
+    be one bf16 step (the fp32 product landed on a tie the exact product is not on) and rare.  Counts
+    are accumulated in g.double_rounding = [differing elements, compared elements]."""
+    if not hasattr(g, "double_rounding"):
+        g.double_rounding = [0, 0]
+    g.double_rounding[1] += int(got.size)
+    if _is_pow2(scale):
+        assert np.array_equal(got, want), "expanded %s rows must be exact for a power-of-two scale" % what
+        return
+    diff = got != want
+    n = int(diff.sum())
+    g.double_rounding[0] += n
+    if n:
+        step = np.abs(got[diff].astype(np.int32) - want[diff].astype(np.int32))
+        assert step.max() == 1, "expanded %s rows differ by more than one bf16 step" % what
+        assert n <= 1e-3 * got.size + 2, "expanded %s rows: %d of %d elements differ" % (what, n, got.size)
 
 
 def check_untouched(g):

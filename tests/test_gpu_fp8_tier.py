@@ -28,8 +28,8 @@ def _to_dev(codes):
     return torch.from_numpy(codes).to(DEV)
 
 
-@pytest.mark.parametrize("fuse,pinned,scales", [(True, False, (1 / 64, 1 / 32)), (False, False, (0.013, 0.021)),
-                                                (True, True, (0.013, 0.021))])
+@pytest.mark.parametrize("fuse,pinned,scales", [(True, False, (1 / 64, 1 / 32)), (True, False, (0.013, 0.021)),
+                                                (False, False, (1 / 64, 1 / 32)), (True, True, (0.013, 0.021))])
 def test_expand_8bit_source_pool(fuse, pinned, scales):
     ks, vs = scales
     w = wl.config(3, requests_override=4)
@@ -55,15 +55,24 @@ def test_expand_8bit_source_pool(fuse, pinned, scales):
         g.k_before, g.v_before, g.src_fmt, g.k_scale, g.v_scale = k8, v8, 1, ks, vs
     else:
         # without the fused rotation the call is "expand, then shift in place": the 16-bit value
-        # bf16(fp32(c) * scale) exists in the page before it is rotated, so the reference is the 16-bit
-        # path applied to a pool of exactly those values
-        as16 = lambda c8, sc: orc.bits(torch.from_numpy(orc.e4m3_decode(c8).astype(np.float32) * np.float32(sc)).to(torch.bfloat16))
+        # c * scale exists in the page before it is rotated (exactly, the scales being powers of two
+        # here), so the reference is the 16-bit path applied to a pool of exactly those values
+        def as16(c8, sc):
+            exact = orc.e4m3_decode(c8) * float(np.float32(sc))
+            b16 = torch.from_numpy(exact).to(torch.bfloat16)
+            assert np.array_equal(b16.double().numpy(), exact)
+            return orc.bits(b16)
         g.k_before, g.v_before = as16(k8, ks), as16(v8, vs)
     g.k_after, g.v_after = orc.bits(t.k_pool), orc.bits(t.v_pool)
     g.kn_bits, g.vn_bits = orc.bits(t.k_new), orc.bits(t.v_new)
     gu.check_placement(g)
     asm, kmx, kmean = gu.check_assembled(g, scattered=False)
     assert kmx > 0                                              # rotated keys were compared
+    if fuse:
+        n_diff, n_all = g.double_rounding
+        print("8-bit expansion, scales %r: %d of %d expanded elements differ from the single-rounding "
+              "definition (one bf16 step each)" % (scales, n_diff, n_all))
+        assert n_all > 0 and (n_diff == 0 or not gu._is_pow2(ks))
     mask = np.ones(w.num_pool_pages, bool)
     mask[g.pages] = False
     assert np.all(g.k_after[mask] == gu.POISON) and np.all(g.v_after[mask] == gu.POISON)

@@ -48,13 +48,27 @@ def test_unfused_compose_then_shift_equals_fused():
 
 
 def test_zero_shift_is_bit_copy():
-    """A unit reused at the position it was cached at must come through bit for bit."""
+    """A unit reused at the position it was cached at must come through bit for bit - including signed
+    zeros whose pair partner is negative (a multiply-add by cos = 1, sin = 0 would turn -0.0 into +0.0)
+    and infinities (0 x Inf would give NaN)."""
     shape = wl.ModelShape(32, 8, 128, 64, 500000.0)
     segs = [wl.unit(300, "a", cached_pos=0, recompute=(0,)), wl.unit(200, "b", cached_pos=300, recompute=(0,)), 5]
     w = wl.build_workload("zero", shape, [segs], np.random.default_rng(1))
-    g = gu.run_layer(w, attention=False)
-    asm, mx, mean = gu.check_assembled(g, scattered=False)
-    assert mx == 0.0 and np.all(asm[0].delta == 0)
+    for fuse in (True, False):
+        t = wl.make_tensors(w, device="cuda:0", seed=13)
+        neg0 = torch.tensor(-0.0, dtype=torch.bfloat16, device="cuda:0")
+        t.k_pool[:, :, :, 0:3] = neg0                                   # -0.0 in the first half ...
+        t.k_pool[:, :, :, 64:67] = -t.k_pool[:, :, :, 64:67].abs() - 1  # ... with a negative partner
+        t.k_pool[:, :, :, 70:72] = neg0                                 # -0.0 in the second half, positive partner
+        t.k_pool[:, :, :, 6:8] = t.k_pool[:, :, :, 6:8].abs() + 1
+        t.k_pool[:, :, :, 10] = float("inf")                            # an infinity next to an ordinary partner
+        g = gu.run_layer(w, t=t, fuse=fuse, attention=False, poison=False)
+        asm, mx, mean = gu.check_assembled(g, scattered=False)
+        assert mx == 0.0 and np.all(asm[0].delta == 0)
+        row = shape.num_kv_heads * shape.head_dim
+        dst = g.k_after.reshape(-1, row)[gu.dest_slots(g, 0)][: 500]
+        assert np.all(dst.reshape(500, 8, 128)[:, :, 0:3] == 0x8000) and np.all(dst.reshape(500, 8, 128)[:, :, 70:72] == 0x8000)
+        assert np.all(dst.reshape(500, 8, 128)[:, :, 10] == 0x7f80)
 
 
 def test_uniform_softmax_lse_and_mean():
@@ -136,22 +150,125 @@ def test_host_buffer_entry_point_matches_device_calls():
     assert torch.equal(lh, g.lse.cpu())
 
 
-@pytest.mark.parametrize("idx,n_random", [(4, 1024), (5, 1024)])
-def test_full_size_sampled(idx, n_random):
+@pytest.mark.parametrize("idx,layer,n_random", [(4, 0, 4096), (4, 15, 4096), (4, 31, 4096), (5, 5, 4096)])
+def test_full_size_sampled(idx, layer, n_random):
     """Configurations too large for the oracle in full: gather compared in full (bit-exact V, block
     table, exact K rows, tolerance on rotated K), attention on the first and last q tile of every
-    request plus random rows."""
+    checked request plus n_random random (request, row, head) triples.  Config 4 is checked on its
+    first, middle and last layer (each layer has its own K / V / Q draw)."""
     w = wl.config(idx)
-    g = gu.run_layer(w, layer=idx)
+    g = gu.run_layer(w, layer=layer)
     assert g.status == 0
     gu.check_placement(g)
     gu.check_untouched(g)
-    rng = np.random.default_rng(idx)
-    reqs = range(w.batch) if idx == 4 else sorted(rng.choice(w.batch, size=8, replace=False).tolist())
+    rng = np.random.default_rng(100 * idx + layer)
+    reqs = list(range(w.batch)) if idx == 4 else sorted(rng.choice(w.batch, size=8, replace=False).tolist())
     asm, kmx, kmean = gu.check_assembled(g, requests=reqs)
     tile_tokens = 128 // (w.shape.num_q_heads // w.shape.num_kv_heads)
-    rows = {r: gu.sample_rows(w, r, rng, n_random // len(list(reqs)), tile_tokens) for r in reqs}
+    rows = {r: gu.sample_rows(w, r, rng, -(-n_random // len(reqs)), tile_tokens) for r in reqs}
+    assert sum(len(v[0]) for v in rows.values()) >= n_random
     gu.check_attention(g, asm, rows_by_request=rows)
+
+
+def _uniform_softmax_exact(w, seed):
+    """K == 0 everywhere: every visible key gets the same weight, so LSE = ln(p + 1) and O = (sum of the
+    visible V rows) / (p + 1) whatever the tiling - a dropped, doubled or wrongly masked key or page
+    shows up directly.  V rows are one-hot (cached: by slot, fresh: by row index), so the sums are small
+    integers.  The expected values are prefix sums over the oracle's assembled V; no oracle attention is
+    needed, so this runs at any length."""
+    dev = "cuda:0"
+    t = wl.make_tensors(w, device=dev, seed=seed)
+    D = w.shape.head_dim
+    t.k_pool.zero_(); t.k_new.zero_()
+    sl = torch.arange(w.num_pool_pages * w.shape.page_size, device=dev)
+    v = torch.nn.functional.one_hot(sl % D, D).to(torch.bfloat16)               # V[slot] = e_(slot mod D)
+    t.v_pool.copy_(v.view(w.num_pool_pages, w.shape.page_size, 1, D).expand_as(t.v_pool))
+    jq = torch.arange(w.n_q, device=dev)
+    vn = torch.nn.functional.one_hot((jq * 5 + 3) % D, D).to(torch.bfloat16)    # V_new[j] = e_((5j + 3) mod D)
+    t.v_new.copy_(vn.view(w.n_q, 1, D).expand_as(t.v_new))
+    g = gu.run_layer(w, t=t, poison=False)
+    assert g.status == 0
+    gu.check_placement(g)
+    asm, _, _ = gu.check_assembled(g)
+    gq = w.shape.num_q_heads // w.shape.num_kv_heads
+    worst_lse = worst_o = 0.0
+    for r, a in asm.items():
+        j0, j1 = int(w.recompute_off[r]), int(w.recompute_off[r + 1])
+        if j1 == j0:
+            continue
+        pos = w.recompute_pos[j0:j1].astype(np.int64)
+        prefix = np.cumsum(orc.bf16_bits_to_f64(a.v_bits), axis=0)              # [T, H_kv, D]: sum of V[0..p]
+        want = prefix[pos] / (pos + 1.0)[:, None, None]                         # [n, H_kv, D]
+        want = np.repeat(want, gq, axis=1)                                      # query head h reads KV head h // g
+        got = g.out_f[j0:j1]
+        err = np.abs(got - want) - (np.abs(want) * 2.0 ** -8 + 1e-6)           # exact up to the final bf16 rounding
+        worst_o = max(worst_o, float(err.max()))
+        lse_err = np.abs(g.lse_f[j0:j1] - np.log(pos + 1.0)[:, None])
+        worst_lse = max(worst_lse, float(lse_err.max()))
+    assert worst_lse < 2e-4, "LSE differs from ln(p + 1) by %.3g" % worst_lse
+    assert worst_o <= 0.0, "O differs from the mean of the visible V rows by %.3g beyond rounding" % worst_o
+    return g
+
+
+def test_uniform_softmax_exact_on_one_full_length_request():
+    """One request of config 4 in full (33 024 tokens, all 2 304 query rows, 258 key steps per work item,
+    two work items per thread block): the path the headline number takes, checked exactly."""
+    w = wl.config(4, requests_override=1)
+    assert int(w.seq_len[0]) == 33024 and w.n_q == 2304
+    g = _uniform_softmax_exact(w, seed=41)
+    assert g.plan.info.n_attn_items == 36 * 8                       # no split along the keys
+
+
+def test_uniform_softmax_exact_on_scattered_rows_with_eight_heads_per_group():
+    """Requests shaped like config 5: 8 query heads per KV head (16 tokens per tile), recompute rows
+    scattered inside the cached units, uncached units recomputed in full."""
+    w = wl.config(5, requests_override=3)
+    uncached = [u for u in range(len(w.unit_len)) if w.unit_page_off[u + 1] == w.unit_page_off[u]]
+    assert uncached and w.shape.num_q_heads // w.shape.num_kv_heads == 8
+    _uniform_softmax_exact(w, seed=42)
+
+
+@pytest.mark.parametrize("n_requests", [1, 3])
+def test_needles_at_long_context_around_page_step_and_ring_boundaries(n_requests):
+    """Keys with an overwhelming logit at positions just before / at / after a page boundary (multiples
+    of 64), a 128-key step boundary and a wrap of the kernel's four-slot K/V ring (every 256 keys), more
+    than 32 K tokens into the context.  A query row at position p must see exactly the needles at
+    positions <= p: with k visible needles each gets weight 1/k in its own output column, an invisible
+    one exactly 0.  One request is split along the keys (too few work items for the GPU), three are not."""
+    shape = wl.ModelShape(32, 8, 128, 64, 500000.0)
+    rng = np.random.default_rng(6)
+    ctx = 32768 + 700
+    lo, hi = 32768 - 200, 32768 + 200                                   # recomputed window inside the cached unit
+    reqs = [[5, wl.unit(ctx, ("ctx", r), recompute=range(lo - 5, hi - 5)), 40] for r in range(n_requests)]
+    w = wl.build_workload("needles", shape, reqs, rng)
+    needles = [32703, 32704, 32705, 32767, 32768, 32769, 32831, 32832, 32895, 32896, 32897]
+    dev = "cuda:0"
+    t = wl.make_tensors(w, device=dev, seed=8)
+    t.k_pool.zero_(); t.v_pool.zero_(); t.k_new.zero_(); t.v_new.zero_()
+    t.q.zero_(); t.q[:, :, 0] = 8.0
+    for r in range(n_requests):
+        j0, j1 = int(w.recompute_off[r]), int(w.recompute_off[r + 1])
+        pos = w.recompute_pos[j0:j1]
+        for i, n in enumerate(needles):
+            j = j0 + int(np.searchsorted(pos, n))
+            assert pos[j - j0] == n
+            t.k_new[j, :, 0] = 64.0
+            t.v_new[j, :, 1 + i] = 1.0
+    g = gu.run_layer(w, t=t, poison=True)
+    assert g.status == 0
+    items = g.plan.info.n_attn_items
+    assert (items < 148) == (n_requests == 1)
+    for r in range(n_requests):
+        j0, j1 = int(w.recompute_off[r]), int(w.recompute_off[r + 1])
+        pos = w.recompute_pos[j0:j1]
+        seen = np.searchsorted(np.array(needles), pos, side="right")            # needles at positions <= p
+        for i in range(len(needles)):
+            col = g.out_f[j0:j1, :, 1 + i]
+            vis = seen > i
+            assert np.all(col[~vis] == 0.0), (r, needles[i])
+            want = 1.0 / seen[vis]
+            assert np.all(np.abs(col[vis] - want[:, None]) <= want[:, None] * 2.0 ** -7), (r, needles[i])
+        assert np.all(g.out_f[j0:j1][seen == 0] == 0.0)
 
 
 def _retention_workloads():

@@ -145,3 +145,29 @@ def test_source_offset_and_target_stride_in_host_plan():
     assert tb.plan_create_status(bad) == tb.INVALID_ARG
     bad = copy.deepcopy(w); bad.unit_target_stride = i32([2])
     assert tb.plan_create_status(bad) == tb.INVALID_ARG
+
+
+def test_capture_descriptor_validation_and_row_count():
+    """Units marked for capture by tessera_extend_write: page count, full recomputation, page clashes."""
+    shape = wl.ModelShape(32, 8, 128, 64, 500000.0)
+    i32 = lambda x: np.asarray(x, np.int32)
+    w0 = wl.build_workload("cap", shape, [[wl.unit(100, "a", recompute=(0, 1)), wl.unit(70, "b", cached=False), 3]],
+                           np.random.default_rng(1), spare_pages=8)
+    used = -(-int(w0.seq_len[0]) // 64)
+    spare = w0.free_pages[used:].tolist()
+
+    def with_capture(off, pages, pool=0):
+        w = copy.copy(w0)
+        w.unit_retain_page_off, w.unit_retain_pages, w.retain_pool_pages = i32(off), i32(pages), pool
+        return w
+
+    ok = with_capture([0, 0, 2], spare[:2])
+    plan = tb.Plan(ok, host_only=True)
+    assert plan.info.retained_tokens == 70
+    assert tb.plan_create_status(with_capture([0, 0, 2], [0, 1], pool=2)) == tb.OK                 # separate cache pool
+    assert tb.plan_create_status(with_capture([0, 2, 2], spare[:2])) == tb.INVALID_ARG             # unit a is not fully recomputed
+    assert tb.plan_create_status(with_capture([0, 0, 1], spare[:1])) == tb.INVALID_ARG             # 70 tokens need 2 pages
+    assert tb.plan_create_status(with_capture([0, 0, 2], [int(w0.unit_pages[0]), spare[0]])) == tb.PAGE_OUT_OF_RANGE   # a source page
+    assert tb.plan_create_status(with_capture([0, 0, 2], [int(w0.free_pages[0]), spare[0]])) == tb.PAGE_OUT_OF_RANGE   # a destination page
+    assert tb.plan_create_status(with_capture([0, 0, 2], [spare[0], spare[0]])) == tb.PAGE_OUT_OF_RANGE                # listed twice
+    assert tb.plan_create_status(with_capture([0, 0, 2], [0, 2], pool=2)) == tb.PAGE_OUT_OF_RANGE                      # outside the cache pool

@@ -136,6 +136,37 @@ def test_paper_position_example_negative_shift():
         assert np.max(np.abs(direct - a0.k[p, 0])) < 1e-10
 
 
+def test_fresh_keys_handed_over_unrotated_are_rotated_for_their_positions():
+    """Sec. 6.1: the forward path captures pre-RoPE keys; Sec. 5.3: the request itself sees them rotated
+    for their positions.  With fresh_k_raw the oracle's assembled key at a recomputed position p must be
+    the library rotary routine applied to the raw key at position p (every head), a bit copy at p = 0,
+    and cached rows must not change."""
+    from transformers.models.llama.modeling_llama import apply_rotary_pos_emb
+    shape = wl.ModelShape(4, 2, 32, 8, 10000.0)
+    w = wl.build_workload("raw", shape, [[3, wl.unit(20, "a", cached_pos=4, recompute=(0, 7)), wl.unit(9, "b", cached=False), 2]],
+                          np.random.default_rng(4))
+    t = wl.make_tensors(w, seed=6)
+    kb, vb, knb, vnb = (orc.bits(x) for x in (t.k_pool, t.v_pool, t.k_new, t.v_new))
+    plain = orc.assemble(w, 0, kb, vb, knb, vnb)
+    raw = orc.assemble(w, 0, kb, vb, knb, vnb, fresh_k_raw=True)
+    D, theta = 32, 10000.0
+    inv = 1.0 / (theta ** (np.arange(0, D, 2, dtype=np.float64) / D))
+    k_new = orc.bf16_bits_to_f64(knb)                                        # [n_q, H_kv, D]
+    fresh = np.zeros(int(w.seq_len[0]), bool)
+    for j, p in enumerate(w.recompute_pos.tolist()):
+        fresh[p] = True
+        emb = np.concatenate([p * inv, p * inv])[None, None, None]
+        cos, sin = torch.from_numpy(np.cos(emb)), torch.from_numpy(np.sin(emb))
+        x = torch.from_numpy(k_new[j][None, :, None, :])                      # [1, heads, 1, D]
+        want, _ = apply_rotary_pos_emb(x, x, cos[0], sin[0])
+        assert np.max(np.abs(want[0, :, 0].numpy() - raw.k[p])) < 1e-12, p
+        assert raw.delta[p] == p and raw.k_exact[p] == (1 if p == 0 else 0)
+        assert np.array_equal(raw.v_bits[p], vnb[j])
+    assert fresh[0] and np.array_equal(raw.k[0], k_new[0])                    # position 0: untouched
+    assert np.array_equal(raw.k[~fresh], plain.k[~fresh]) and np.array_equal(raw.v_bits, plain.v_bits)
+    assert np.abs(raw.k[fresh][1:] - plain.k[fresh][1:]).max() > 0.1          # and it really differs from the rotated-input reading
+
+
 # ---------------------------------------------------------------------- placement
 
 def _placement_by_hand(w):
@@ -171,6 +202,100 @@ def test_placement(make):
     assert sorted(fresh[fresh >= 0]) == list(range(w.n_q))
     # destination pages never alias source pages
     assert not (set(pages.tolist()) & set(w.unit_pages.tolist()))
+
+
+def _read_placement_golden():
+    """Parses tests/golden/placement_slots.txt into a list of (name, Workload, expected dict)."""
+    cases, cur = [], None
+    for line in open(os.path.join(GOLDEN, "placement_slots.txt")):
+        line = line.split("#")[0].strip()
+        if not line:
+            continue
+        key, *rest = line.split()
+        if key == "case":
+            cur = {"name": rest[0], "units": []}
+            cases.append(cur)
+        elif key == "unit":
+            k = rest.index("pages")
+            cur["units"].append(([int(x) for x in rest[:k]], [int(x) for x in rest[k + 1:]]))
+        else:
+            cur[key] = [int(x) for x in rest]
+    out = []
+    i32 = lambda x: np.asarray(x, np.int32)
+    for c in cases:
+        B = c["B"][0]
+        shape = wl.ModelShape(4, 2, 64, B, 1e4)
+        ulen = [u[0][0] for u in c["units"]]
+        pages = [p for u in c["units"] for p in u[1]]
+        poff = np.cumsum([0] + [len(u[1]) for u in c["units"]])
+        w = wl.Workload(name=c["name"], shape=shape, seq_len=i32(c["seq_len"]), unit_off=i32([0, len(ulen)]),
+                        unit_len=i32(ulen), unit_cached_pos=i32([0] * len(ulen)), unit_cached_stride=i32([1] * len(ulen)),
+                        unit_target_pos=i32([u[0][1] for u in c["units"]]), unit_page_off=i32(poff), unit_pages=i32(pages),
+                        recompute_off=i32([0, len(c["recompute"])]), recompute_pos=i32(c["recompute"]),
+                        free_pages=i32(c["free"]), num_pool_pages=max(pages + c["free"]) + 1,
+                        unit_src_offset=i32([u[0][2] for u in c["units"]]))
+        out.append((c["name"], w, c))
+    return out
+
+
+def test_placement_against_hand_written_golden():
+    """Literal slot numbers worked out by hand (tests/golden/placement_slots.txt), with and without a
+    source offset: the oracle's slot arithmetic against something that is not its own formula."""
+    cases = _read_placement_golden()
+    assert len(cases) >= 4
+    for name, w, c in cases:
+        st, page_off, pages, src, fresh = orc.placement(w)
+        assert st == 0, name
+        assert pages.tolist() == c["block_table"], name
+        assert src.tolist() == c["src_slot"], name
+        B = w.shape.page_size
+        dst = [int(pages[p // B]) * B + p % B for p in range(int(w.seq_len[0]))]
+        assert dst == c["dst_slot"], name
+        assert [p for p in range(len(fresh)) if fresh[p] >= 0] == c["recompute"], name
+
+
+def test_retained_form_is_the_unrotated_key():
+    """Store side (Sec. 5.3: the miss prefill keeps an unrotated copy for the cache; Sec. 6.1: pre-RoPE
+    keys are captured).  A unit whose keys sit in a request's pages rotated at positions p0 + i, retained
+    with target stride 0 at target position 0, must come out as R(-(p0 + i)) applied to each stored key,
+    i.e. as the key before any rotation: assembling it and rotating back by +(p0 + i) returns the stored
+    key, and the per-token shifts are exactly -(p0 + i)."""
+    shape = wl.ModelShape(4, 2, 16, 4, 100.0)
+    i32 = lambda x: np.asarray(x, np.int32)
+    p0, n = 6, 7                                                     # unit at positions 6..12 of the request
+    w = wl.Workload(name="retain", shape=shape, seq_len=i32([n]), unit_off=i32([0, 1]), unit_len=i32([n]),
+                    unit_cached_pos=i32([p0]), unit_cached_stride=i32([1]), unit_target_pos=i32([0]),
+                    unit_page_off=i32([0, 3]), unit_pages=i32([5, 1, 3]), recompute_off=i32([0, 0]),
+                    recompute_pos=i32([]), free_pages=i32([0, 2]), num_pool_pages=6,
+                    unit_src_offset=i32([p0 % 4]), unit_target_stride=i32([0]))
+    # pool rows are arbitrary bf16 numbers x_i (what the request's pages hold at positions p0 + i);
+    # the retained row must be R(-(p0 + i)) x_i
+    t = wl.make_tensors(w, seed=3)
+    kb, vb = orc.bits(t.k_pool), orc.bits(t.v_pool)
+    none = np.zeros((1, 2 * 16), np.uint16)
+    a = orc.assemble(w, 0, kb, vb, none, none)
+    assert a.delta.tolist() == [-(p0 + i) for i in range(n)]
+    pool = orc.bf16_bits_to_f64(kb).reshape(-1, 2, 16)
+    for i in range(n):
+        si = p0 % 4 + i
+        slot = [5, 1, 3][si // 4] * 4 + si % 4
+        for h in range(2):
+            want = orc.rope_rotate(pool[slot, h], -(p0 + i), 100.0)
+            assert np.max(np.abs(want - a.k[i, h])) < 1e-12
+            back = orc.rope_rotate(a.k[i, h], p0 + i, 100.0)           # rotating forward again returns the stored key
+            assert np.max(np.abs(back - pool[slot, h])) < 1e-12
+        assert np.array_equal(a.v_bits[i], vb.reshape(-1, 2, 16)[slot])
+    # with target stride 1 (the default) the same descriptor shifts every token by the same -p0
+    w1 = wl.Workload(**{**w.__dict__, "unit_target_stride": None})
+    a1 = orc.assemble(w1, 0, kb, vb, none, none)
+    assert a1.delta.tolist() == [-p0] * n
+    # one worked number: pair 0 turns by exactly (shift) radians whatever theta is (w_0 = 1), so for
+    # token 2 (shift -8) element 0 of head 0 is x cos 8 + y sin 8 with (x, y) = (elements 0 and 8)
+    si = p0 % 4 + 2
+    slot = [5, 1, 3][si // 4] * 4 + si % 4
+    x, y = pool[slot, 0, 0], pool[slot, 0, 8]
+    assert abs(a.k[2, 0, 0] - (x * math.cos(8.0) + y * math.sin(8.0))) < 1e-12
+    assert abs(a.k[2, 0, 8] - (y * math.cos(8.0) - x * math.sin(8.0))) < 1e-12
 
 
 def test_placement_rejects_bad_batches():
@@ -380,10 +505,44 @@ def test_assemble_from_8bit_pool_reduces_to_the_16bit_path():
             a8 = orc.assemble(w, r, k8, v8, knb, vnb, src_fmt=1, k_scale=scale, v_scale=scale)
             assert np.array_equal(a16.v_bits, a8.v_bits) and np.array_equal(a16.k, a8.k)
             assert np.array_equal(a16.k_exact, a8.k_exact) and np.array_equal(a16.k_bits, a8.k_bits)
-    # a scale that is not a power of two: the 16-bit row is the float product rounded once more to bf16
+    # a scale that is not a power of two: the 16-bit row is the EXACT product code * float(scale) rounded
+    # once to bf16.  Checked against exact rational arithmetic: the result must be the bf16 neighbour
+    # nearest to the exact product, the even one on a tie.
+    from fractions import Fraction
     a8 = orc.assemble(w, 0, k8, v8, knb, vnb, src_fmt=1, k_scale=0.3, v_scale=0.7)
     st, _, _, src_slot, fresh = orc.placement(w)
     row = w.shape.num_kv_heads * w.shape.head_dim
     p = next(p for p in range(int(w.seq_len[0])) if fresh[p] < 0)
-    want = (orc.e4m3_decode(v8.reshape(-1, row)[src_slot[p]]).astype(np.float32) * np.float32(0.7))
-    assert np.array_equal(a8.v_bits[p].ravel(), orc.bits(torch.from_numpy(want).to(torch.bfloat16)))
+    codes = v8.reshape(-1, row)[src_slot[p]]
+    sc = Fraction(float(np.float32(0.7)))
+    got = orc.bf16_bits_to_f64(a8.v_bits[p].ravel())
+    for c, gv, gb in zip(codes.tolist(), got.tolist(), a8.v_bits[p].ravel().tolist()):
+        exact = Fraction(float(orc.e4m3_decode(np.array([c], np.uint8))[0])) * sc
+        if exact == 0:
+            assert gv == 0.0
+            continue
+        up = orc.bf16_bits_to_f64(np.array([gb + 1], np.uint16))[0]      # next bf16 away from zero
+        dn = orc.bf16_bits_to_f64(np.array([gb - 1], np.uint16))[0]      # next bf16 towards zero
+        err = abs(Fraction(gv) - exact)
+        for nb in (up, dn):
+            e2 = abs(Fraction(float(nb)) - exact)
+            assert err < e2 or (err == e2 and gb % 2 == 0), (c, gv, nb)
+
+
+def test_f64_to_bf16_single_rounding():
+    """The oracle's double -> bf16 rounding against the library's float -> bfloat16 conversion on values
+    that are floats already (one rounding either way), plus the cases where rounding a double through
+    float first would go wrong (a double just above / below a bf16 midpoint)."""
+    rng = np.random.default_rng(3)
+    x = (rng.standard_normal(20000) * np.exp(rng.uniform(-30, 30, 20000))).astype(np.float32)
+    want = orc.bits(torch.from_numpy(x).to(torch.bfloat16))
+    assert np.array_equal(orc.f64_to_bf16_bits(x.astype(np.float64)), want)
+    # 1 + 2^-8 is the midpoint between bf16 1.0 (0x3f80, even) and 1 + 2^-7 (0x3f81)
+    mid = 1.0 + 2.0 ** -8
+    assert orc.f64_to_bf16_bits(np.array([mid, mid + 2.0 ** -40, mid - 2.0 ** -40])).tolist() == [0x3f80, 0x3f81, 0x3f80]
+    # 1 + 3 * 2^-8 is the midpoint between 0x3f81 (odd) and 0x3f82 (even): the tie goes up to the even one
+    assert orc.f64_to_bf16_bits(np.array([1.0 + 3 * 2.0 ** -8])).tolist() == [0x3f82]
+    # rounding through float first would turn mid + 2^-40 into the exact midpoint and lose the tie
+    assert np.float32(mid + 2.0 ** -40) == np.float32(mid)
+    assert orc.f64_to_bf16_bits(np.array([0.0, -0.0, np.inf, -np.inf, 2.0 ** -140, -1.5])).tolist() == \
+        [0x0000, 0x8000, 0x7f80, 0xff80, 0x0000, 0xbfc0]
