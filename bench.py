@@ -403,9 +403,11 @@ def fp8_tier_record(w, dev, steps, warmup, peaks):
 
 
 def host_tier_record(w, dev, steps, warmup):
-    """Local-hit tier: the cached units live in a pinned host-memory pool and are composed into the
-    requests' device pages.  `zero_copy`: the gather kernel reads the host pool over the link
-    (tessera_kv_compose_from).  Bytes over the link = K and V rows of every cached token."""
+    """Local-hit tier: the cached units live in a pinned host-memory pool.  One layer = compose from that
+    pool + fresh-row scatter + attention.  `zero_copy_then_attention`: the gather kernel reads the host
+    pool over the link (tessera_kv_compose_from), attention follows.  `overlapped`: a small reader launch
+    pulls chunk c + 1 while scatter + attention of chunk c run (tessera_composed_prefill_host_tier), for
+    bf16 and for e4m3 units.  Bytes over the link = K and V rows of every cached token."""
     import torch
     from paper_2609_32999_b200 import binding as tb
     from paper_2609_32999_b200 import workloads as wl
@@ -414,22 +416,61 @@ def host_tier_record(w, dev, steps, warmup):
     plan = tb.Plan(w2)
     t = wl.make_tensors(w, layer=0, device=dev, seed=wl.BASE_SEED)
     host_k, host_v = t.k_pool.cpu().pin_memory(), t.v_pool.cpu().pin_memory()
+    sh = w.shape
+    out = torch.empty(w.n_q, sh.num_q_heads, sh.head_dim, dtype=torch.bfloat16, device=dev)
+    lse = torch.empty(w.n_q, sh.num_q_heads, dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
-    link_bytes = w.cached_tokens * w.shape.num_kv_heads * w.shape.head_dim * 2 * 2
-    rec = {"workload": w.name, "cached_tokens": int(w.cached_tokens), "link_bytes_per_layer": int(link_bytes), "steps": steps}
+    row_bytes = sh.num_kv_heads * sh.head_dim * 2 * 2
+    rec = {"workload": w.name, "cached_tokens": int(w.cached_tokens), "steps": steps}
     launches0 = tb.launch_count()
-    ms = []
-    for i in range(warmup + steps):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
+
+    def timed(fn):
+        ms = []
+        for i in range(warmup + steps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= warmup:
+                ms.append(a.elapsed_time(b))
+        return sum(ms) / len(ms)
+
+    m_gather = timed(lambda: plan.kv_compose_from(host_k, host_v, t.k_pool, t.v_pool))
+    m_attn = timed(lambda: plan.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, out, lse))
+
+    def zero_copy_layer():
         plan.kv_compose_from(host_k, host_v, t.k_pool, t.v_pool)
-        b.record(stream)
-        torch.cuda.synchronize()
-        if i >= warmup:
-            ms.append(a.elapsed_time(b))
-    m = sum(ms) / len(ms)
-    rec["zero_copy"] = {"ms_per_layer": m, "link_GBps": link_bytes / m / 1e6}
+        plan.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, out, lse)
+
+    m_zero = timed(zero_copy_layer)
+    link_bytes = w.cached_tokens * row_bytes
+    rec["zero_copy_then_attention"] = {"ms_per_layer": m_zero, "gather_ms": m_gather, "attention_ms": m_attn,
+                                       "link_bytes_per_layer": int(link_bytes), "link_GBps_during_gather": link_bytes / m_gather / 1e6}
+    m_over = timed(lambda: plan.composed_prefill_host_tier(host_k, host_v, t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, out, lse))
+    rec["overlapped"] = {"ms_per_layer": m_over, "link_GBps": link_bytes / m_over / 1e6,
+                         "saved_ms_vs_sequential": m_zero - m_over,
+                         # share of the attention time that ran under the transfer
+                         "attention_hidden_frac": max(0.0, min(1.0, (m_zero - m_over) / m_attn))}
+    # e4m3 units: half the bytes over the link
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(wl.BASE_SEED)
+    shape8 = tuple(t.k_pool.shape)
+    draw8 = lambda: (torch.randint(0, 0x78, shape8, dtype=torch.uint8, generator=gen)
+                     | (torch.randint(0, 2, shape8, dtype=torch.uint8, generator=gen) << 7)).pin_memory()
+    k8, v8 = draw8(), draw8()
+
+    def zero_copy_layer8():
+        plan.kv_compose_from_fp8(k8, v8, 1 / 32, 1 / 32, t.k_pool, t.v_pool)
+        plan.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, out, lse)
+
+    m_zero8 = timed(zero_copy_layer8)
+    m8 = timed(lambda: plan.composed_prefill_host_tier(k8, v8, t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, out, lse,
+                                                       src_format=1, k_scale=1 / 32, v_scale=1 / 32))
+    rec["e4m3_units"] = {"sequential_ms_per_layer": m_zero8, "overlapped_ms_per_layer": m8,
+                         "link_bytes_per_layer": int(link_bytes // 2), "link_GBps": link_bytes / 2 / m8 / 1e6}
     rec["gpu_launches"] = tb.launch_count() - launches0
+    assert plan.status() == 0
     plan.destroy()
     return rec
 
@@ -715,7 +756,7 @@ def main():
             torch.cuda.empty_cache()
         line["per_config"] = per_config
         w4 = w if args.config == 4 else rank_workload(4, rank, None, None)
-        line["host_tier"] = host_tier_record(w4, dev, 3, 2)
+        line["host_tier"] = [host_tier_record(w4, dev, 3, 2), host_tier_record(rank_workload(3, rank, None, None), dev, 5, 2)]
         torch.cuda.empty_cache()
         line["fp8_tier"] = fp8_tier_record(w4, dev, 8, 3, peaks)
     print(json.dumps(line))

@@ -301,6 +301,32 @@ TESSERA_API int32_t tessera_composed_prefill_host(tessera_plan *plan, void *k_po
                                       void *out_host, float *lse_host, void *stream);
 
 /*
+ * The per-layer path when the cached units sit in the node's PINNED HOST-MEMORY cache (Sec. 5.3
+ * "Preparing cache hits": a local hit is copied from the pinned host cache into the request's KV slots
+ * while the engine keeps working on what is already prepared).  The plan must have been created with
+ * desc.num_source_pages > 0.  The batch is cut into chunks of whole requests.  For each chunk a reader
+ * launch of the gather kernel - `reader_blocks` thread blocks walking the chunk's copy list on a side
+ * stream of the plan - pulls the rows over the interconnect straight into their destination slots, keys
+ * rotated on the way (no staging buffer is needed: the bound on extra device memory is zero); when a
+ * chunk has arrived, its fresh-row scatter + attention run on `stream` with a grid that leaves the
+ * reader's SMs free, so attention of chunk c overlaps the transfer of chunk c + 1.  Results are
+ * bit-identical to tessera_kv_compose_from + tessera_partial_prefill_attn.
+ *   k_src_host, v_src_host  host, pinned and device-addressable (cudaHostAlloc / cudaHostRegister),
+ *                           [num_source_pages][page_size][H_kv][D], 16-byte aligned, never written; bf16
+ *                           when src_format is 0, e4m3 codes standing for code * k_scale / v_scale when
+ *                           src_format is 1 (the scales are ignored for format 0)
+ *   q, k_new, v_new, out, lse   device, as in tessera_partial_prefill_attn
+ *   reader_blocks           thread blocks (of 256 threads) of the reader; 0 = 16; at most half the SM count
+ * All work is enqueued on `stream` and on the side stream; the call returns without waiting.  The host
+ * pools must stay valid and unchanged until `stream` has drained.
+ */
+TESSERA_API int32_t tessera_composed_prefill_host_tier(tessera_plan *plan, const void *k_src_host, const void *v_src_host,
+                                                       int32_t src_format, float k_scale, float v_scale,
+                                                       void *k_pool, void *v_pool, const void *q, const void *k_new,
+                                                       const void *v_new, void *out, float *lse, int32_t reader_blocks,
+                                                       void *stream);
+
+/*
  * In-place RoPE shift for callers that cannot allocate device memory.  (The paper has no
  * counterpart; this is a service entry of this library.)  Some callers run where cudaMalloc is off
  * limits: inside a serving engine that owns the whole device through its own memory pool, in a

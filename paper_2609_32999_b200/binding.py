@@ -56,7 +56,7 @@ class PlanInfo(ctypes.Structure):
 
 EXPORTS = ["tessera_plan_create", "tessera_plan_destroy", "tessera_plan_block_table", "tessera_plan_get_info",
            "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_kv_compose_from_fp8", "tessera_kv_retain_fp8", "tessera_rope_shift", "tessera_rope_fresh", "tessera_extend_write", "tessera_partial_prefill_attn",
-           "tessera_composed_prefill_host", "tessera_rope_shift_static", "tessera_selftest_bounded_wait", "tessera_last_error",
+           "tessera_composed_prefill_host", "tessera_composed_prefill_host_tier", "tessera_rope_shift_static", "tessera_selftest_bounded_wait", "tessera_last_error",
            "tessera_launch_count"]
 
 _vp = ctypes.c_void_p
@@ -75,6 +75,8 @@ _lib.tessera_rope_fresh.argtypes = [_vp, _vp, _vp, _vp]
 _lib.tessera_extend_write.argtypes = [_vp] * 9
 _lib.tessera_partial_prefill_attn.argtypes = [_vp] * 9
 _lib.tessera_composed_prefill_host.argtypes = [_vp] * 9
+_lib.tessera_composed_prefill_host_tier.argtypes = [_vp, _vp, _vp, ctypes.c_int32, ctypes.c_float, ctypes.c_float,
+                                                    _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_int32, _vp]
 _lib.tessera_rope_shift_static.argtypes = [ctypes.POINTER(ModelCfg), _vp, ctypes.c_int64, _vp, _vp, ctypes.c_int32,
                                            _I32P, ctypes.c_int32, _vp]
 _lib.tessera_selftest_bounded_wait.argtypes = [ctypes.c_int64, _I32P, ctypes.POINTER(ctypes.c_int64), _vp]
@@ -222,6 +224,16 @@ class Plan:
         _check(_lib.tessera_composed_prefill_host(self._h, _dev(k_pool), _dev(v_pool), _dev(q_host),
                                                   _dev(k_new_host), _dev(v_new_host), _dev(out_host),
                                                   _dev(lse_host), _stream(stream)))
+
+    def composed_prefill_host_tier(self, k_src_host, v_src_host, k_pool, v_pool, q, k_new, v_new, out, lse=None,
+                                   src_format: int = 0, k_scale: float = 1.0, v_scale: float = 1.0,
+                                   reader_blocks: int = 0, stream=None) -> None:
+        """Cached units in pinned host pools (bf16, or e4m3 codes with src_format=1), pulled over the link
+        chunk by chunk by a small reader launch while attention of the chunks already there runs."""
+        _check(_lib.tessera_composed_prefill_host_tier(self._h, _dev(k_src_host), _dev(v_src_host), int(src_format),
+                                                       float(k_scale), float(v_scale), _dev(k_pool), _dev(v_pool),
+                                                       _dev(q), _dev(k_new), _dev(v_new), _dev(out), _dev(lse),
+                                                       int(reader_blocks), _stream(stream)))
 
     def destroy(self) -> None:
         if self._h:

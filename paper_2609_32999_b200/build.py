@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtessera.so")
 SOURCES = ["api.cu", "plan.cu", "gather_rope.cu", "kv_fp8.cu", "attn_tc.cu",
-           "rope_shift_static.cu", "selftest.cu"]
+           "rope_shift_static.cu", "host_tier.cu", "selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 

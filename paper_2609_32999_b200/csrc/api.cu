@@ -137,10 +137,10 @@ bool misaligned(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) !=
 
 // Fresh-row scatter + attention of the whole batch (chunk < 0) or of one request chunk.
 int32_t attention(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, const void *k_new,
-                  const void *v_new, void *out, float *lse, int chunk, cudaStream_t st) {
+                  const void *v_new, void *out, float *lse, int chunk, cudaStream_t st, int max_blocks = 0) {
     TS_CUDA(launch_scatter_fresh(pl, k_pool, v_pool, k_new, v_new, chunk, st));
     std::string err;
-    cudaError_t e = launch_attn_tc(pl, k_pool, v_pool, q, out, lse, chunk, st, &err);
+    cudaError_t e = launch_attn_tc(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, st, &err);
     if (e != cudaSuccess) return set_error(TESSERA_CUDA_ERROR, "tcgen05 attention launch: " + err + " / " + cudaGetErrorString(e));
     return TESSERA_OK;
 }
@@ -166,8 +166,14 @@ int32_t ensure_pipeline(tessera_plan *pl) {
 
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
-// Lets entry points defined in other files record the calling thread's error text.
+// Lets entry points defined in other files record the calling thread's error text, run scatter +
+// attention of one request chunk (optionally on a capped grid), and create the plan's side streams.
 int32_t api_set_error(int32_t code, const std::string &msg) { return set_error(code, msg); }
+int32_t api_attention(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, const void *k_new,
+                      const void *v_new, void *out, float *lse, int chunk, int max_blocks, cudaStream_t st) {
+    return attention(pl, k_pool, v_pool, q, k_new, v_new, out, lse, chunk, st, max_blocks);
+}
+int32_t api_ensure_pipeline(tessera_plan *pl) { return ensure_pipeline(pl); }
 
 }  // namespace tessera
 

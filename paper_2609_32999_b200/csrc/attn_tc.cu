@@ -666,7 +666,7 @@ attn_combine_kernel(const CombineItem *__restrict__ items, const AttnTile *__res
 
 template <int D, int kMaxPages>
 cudaError_t launch_attn_tc_d(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
-                             float *lse, int chunk, cudaStream_t st, std::string *err) {
+                             float *lse, int chunk, int max_blocks, cudaStream_t st, std::string *err) {
     const AttnWork *work = chunk < 0 ? pl->dev.work : pl->dev.work_chunked + pl->chunk_work_off[chunk];
     const size_t n_work = chunk < 0 ? pl->work.size() : (size_t)(pl->chunk_work_off[chunk + 1] - pl->chunk_work_off[chunk]);
     if (n_work == 0) return cudaSuccess;
@@ -683,7 +683,8 @@ cudaError_t launch_attn_tc_d(const tessera_plan *pl, void *k_pool, void *v_pool,
     const DeviceTables &d = pl->dev;
     const float scale_log2 = pl->sm_scale * 1.4426950408889634f;
     // persistent: one thread block per SM (fewer when the list is shorter)
-    const unsigned grid = (unsigned)std::min<size_t>(n_work, (size_t)pl->num_sms);
+    const int sms = max_blocks > 0 ? std::min(max_blocks, pl->num_sms) : pl->num_sms;
+    const unsigned grid = (unsigned)std::min<size_t>(n_work, (size_t)sms);
     attn_tc_kernel<D, kMaxPages><<<grid, kThreads, Geo<D>::kSmemAlloc, st>>>(
         tq, tk, tv, to, d.tiles, work, (int)n_work, d.q_pos, d.page_off, d.pages, d.seq_len,
         static_cast<__nv_bfloat16 *>(out), lse, Hq, g, Hkv, ps, pl->num_pool_pages, scale_log2, pl->max_parts, d.ws_o, d.ws_ml, d.status);
@@ -705,7 +706,7 @@ cudaError_t launch_attn_tc_d(const tessera_plan *pl, void *k_pool, void *v_pool,
 }  // namespace
 
 cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
-                           float *lse, int chunk, cudaStream_t st, std::string *err) {
+                           float *lse, int chunk, int max_blocks, cudaStream_t st, std::string *err) {
     if (pl->n_q == 0 || pl->work.empty()) return cudaSuccess;
     const int D = pl->cfg.head_dim, ps = pl->cfg.page_size, g = pl->cfg.num_q_heads / pl->cfg.num_kv_heads;
     if ((D != 64 && D != 128) || (ps != 8 && ps != 16 && ps != 32 && ps != 64 && ps != 128) || g > 16) {
@@ -713,10 +714,10 @@ cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, c
         return cudaErrorNotSupported;
     }
     if (ps == 8)
-        return D == 128 ? launch_attn_tc_d<128, 16>(pl, k_pool, v_pool, q, out, lse, chunk, st, err)
-                        : launch_attn_tc_d<64, 16>(pl, k_pool, v_pool, q, out, lse, chunk, st, err);
-    return D == 128 ? launch_attn_tc_d<128, 8>(pl, k_pool, v_pool, q, out, lse, chunk, st, err)
-                    : launch_attn_tc_d<64, 8>(pl, k_pool, v_pool, q, out, lse, chunk, st, err);
+        return D == 128 ? launch_attn_tc_d<128, 16>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, st, err)
+                        : launch_attn_tc_d<64, 16>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, st, err);
+    return D == 128 ? launch_attn_tc_d<128, 8>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, st, err)
+                    : launch_attn_tc_d<64, 8>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, st, err);
 }
 
 }  // namespace tessera

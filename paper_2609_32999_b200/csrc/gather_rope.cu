@@ -98,14 +98,17 @@ template <int D, bool DO_V, bool ROTATE, bool IN_PLACE, bool INTERLEAVED>
 __global__ void __launch_bounds__(kThreads)
 gather_rope_kernel(const uint4 *k_src, const uint4 *v_src, uint4 *k_pool, uint4 *v_pool,
                    const int32_t *__restrict__ g_src, const int32_t *__restrict__ g_dst,
-                   const GatherItem *__restrict__ items, const float2 *__restrict__ rope, int H_kv) {
+                   const GatherItem *__restrict__ items, int n_items, const float2 *__restrict__ rope, int H_kv) {
     constexpr int CPH = D / 16;          // pair-chunks per head
     constexpr int HALF = D / 16;         // distance (in 16-byte chunks) between pair partners
     __shared__ float2 s_rope[kGatherItemTokens * (D / 2)];
     __shared__ int32_t s_src[kGatherItemTokens], s_dst[kGatherItemTokens];
 
-    const GatherItem it = items[blockIdx.x];
     const int tid = threadIdx.x;
+    // one item per thread block in the ordinary launch; a launch with fewer blocks than items (the
+    // host-tier reader, which must leave most SMs to the attention kernel) walks the list
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const GatherItem it = items[item];
     // rows row0, row0 + step, ... of the table; with step = -1 they are staged in ascending order
     const int n_rows = ROTATE ? (it.row_step ? it.count : 1) : 0;
     const int first_row = it.row_step < 0 ? it.row0 - (it.count - 1) : it.row0;
@@ -176,6 +179,8 @@ gather_rope_kernel(const uint4 *k_src, const uint4 *v_src, uint4 *k_pool, uint4 
             stg(k_pool + dsto[u], klo[u]);
             stg(k_pool + dsto[u] + HALF, khi[u]);
         }
+    }
+    __syncthreads();          // the staged rows are rewritten by the next item
     }
 }
 
@@ -304,8 +309,9 @@ extend_write_kernel(uint4 *__restrict__ q, const uint4 *__restrict__ k_raw, cons
 
 template <int D, bool IL>
 cudaError_t launch_gather_d(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
-                            GatherMode mode, const int32_t *g_src, int first_item, int n, cudaStream_t st) {
+                            GatherMode mode, const int32_t *g_src, int first_item, int n, int max_blocks, cudaStream_t st) {
     if (n == 0) return cudaSuccess;
+    const int grid = max_blocks > 0 ? std::min(n, max_blocks) : n;
     auto *kp = static_cast<uint4 *>(k_pool);
     auto *vp = static_cast<uint4 *>(v_pool);
     auto *ks = static_cast<const uint4 *>(k_src);
@@ -315,13 +321,13 @@ cudaError_t launch_gather_d(const tessera_plan *pl, const void *k_src, const voi
     const int H = pl->cfg.num_kv_heads;
     switch (mode) {
         case GatherMode::kCopy:
-            gather_rope_kernel<D, true, false, false, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, g_src, d.g_dst, items, d.rope, H);
+            gather_rope_kernel<D, true, false, false, IL><<<grid, kThreads, 0, st>>>(ks, vs, kp, vp, g_src, d.g_dst, items, n, d.rope, H);
             break;
         case GatherMode::kCopyRotate:
-            gather_rope_kernel<D, true, true, false, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, g_src, d.g_dst, items, d.rope, H);
+            gather_rope_kernel<D, true, true, false, IL><<<grid, kThreads, 0, st>>>(ks, vs, kp, vp, g_src, d.g_dst, items, n, d.rope, H);
             break;
         case GatherMode::kShiftInPlace:
-            gather_rope_kernel<D, false, true, true, IL><<<n, kThreads, 0, st>>>(ks, vs, kp, vp, g_src, d.g_dst, items, d.rope, H);
+            gather_rope_kernel<D, false, true, true, IL><<<grid, kThreads, 0, st>>>(ks, vs, kp, vp, g_src, d.g_dst, items, n, d.rope, H);
             break;
     }
     count_launch();
@@ -331,18 +337,19 @@ cudaError_t launch_gather_d(const tessera_plan *pl, const void *k_src, const voi
 }  // namespace
 
 cudaError_t launch_gather_range(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
-                                GatherMode mode, const int32_t *g_src, int first_item, int n_items, cudaStream_t st) {
+                                GatherMode mode, const int32_t *g_src, int first_item, int n_items, int max_blocks,
+                                cudaStream_t st) {
     const bool il = pl->cfg.rope_pairing == 1;
     if (pl->cfg.head_dim == 128)
-        return il ? launch_gather_d<128, true>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, st)
-                  : launch_gather_d<128, false>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, st);
-    return il ? launch_gather_d<64, true>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, st)
-              : launch_gather_d<64, false>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, st);
+        return il ? launch_gather_d<128, true>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, max_blocks, st)
+                  : launch_gather_d<128, false>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, max_blocks, st);
+    return il ? launch_gather_d<64, true>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, max_blocks, st)
+              : launch_gather_d<64, false>(pl, k_src, v_src, k_pool, v_pool, mode, g_src, first_item, n_items, max_blocks, st);
 }
 
 cudaError_t launch_gather(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
                           GatherMode mode, cudaStream_t st) {
-    return launch_gather_range(pl, k_src, v_src, k_pool, v_pool, mode, pl->dev.g_src, 0, (int)pl->items.size(), st);
+    return launch_gather_range(pl, k_src, v_src, k_pool, v_pool, mode, pl->dev.g_src, 0, (int)pl->items.size(), 0, st);
 }
 
 cudaError_t launch_rope_fresh(const tessera_plan *pl, void *q, void *k_new, cudaStream_t st) {

@@ -98,14 +98,17 @@ template <int D, bool TO_8BIT, bool ROTATE, bool INTERLEAVED>
 __global__ void __launch_bounds__(kThreads)
 kv_fp8_kernel(const void *__restrict__ k_src, const void *__restrict__ v_src, void *__restrict__ k_dst,
               void *__restrict__ v_dst, const int32_t *__restrict__ g_src, const int32_t *__restrict__ g_dst,
-              const GatherItem *__restrict__ items, const float2 *__restrict__ rope, int H_kv, float k_mul, float v_mul) {
+              const GatherItem *__restrict__ items, int n_items, const float2 *__restrict__ rope, int H_kv, float k_mul,
+              float v_mul) {
     constexpr int CPH = D / 16;          // pair-chunks per head
     constexpr int HALF = D / 16;         // distance (in 8-element chunks) between pair partners
     __shared__ float2 s_rope[kGatherItemTokens * (D / 2)];
     __shared__ int32_t s_src[kGatherItemTokens], s_dst[kGatherItemTokens];
 
-    const GatherItem it = items[blockIdx.x];
     const int tid = threadIdx.x;
+    // one item per thread block, or - when launched with fewer blocks than items - a walk through the list
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const GatherItem it = items[item];
     const int n_rows = ROTATE ? (it.row_step ? it.count : 1) : 0;
     const int first_row = it.row_step < 0 ? it.row0 - (it.count - 1) : it.row0;
     for (int i = tid; i < n_rows * (D / 2); i += kThreads) s_rope[i] = rope[(size_t)first_row * (D / 2) + i];
@@ -180,47 +183,50 @@ kv_fp8_kernel(const void *__restrict__ k_src, const void *__restrict__ v_src, vo
             }
         }
     }
+    __syncthreads();          // the staged rows are rewritten by the next item
+    }
 }
 
 template <int D, bool TO_8BIT, bool IL>
 cudaError_t launch_d(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst, bool rotate,
-                     float k_mul, float v_mul, const int32_t *g_src, int first_item, int n, cudaStream_t st) {
+                     float k_mul, float v_mul, const int32_t *g_src, int first_item, int n, int max_blocks, cudaStream_t st) {
     if (n == 0) return cudaSuccess;
+    const int grid = max_blocks > 0 ? (n < max_blocks ? n : max_blocks) : n;
     const DeviceTables &d = pl->dev;
     const GatherItem *items = d.items + first_item;
     const int H = pl->cfg.num_kv_heads;
     if (rotate)
-        kv_fp8_kernel<D, TO_8BIT, true, IL><<<n, kThreads, 0, st>>>(k_src, v_src, k_dst, v_dst, g_src, d.g_dst, items, d.rope, H, k_mul, v_mul);
+        kv_fp8_kernel<D, TO_8BIT, true, IL><<<grid, kThreads, 0, st>>>(k_src, v_src, k_dst, v_dst, g_src, d.g_dst, items, n, d.rope, H, k_mul, v_mul);
     else
-        kv_fp8_kernel<D, TO_8BIT, false, IL><<<n, kThreads, 0, st>>>(k_src, v_src, k_dst, v_dst, g_src, d.g_dst, items, d.rope, H, k_mul, v_mul);
+        kv_fp8_kernel<D, TO_8BIT, false, IL><<<grid, kThreads, 0, st>>>(k_src, v_src, k_dst, v_dst, g_src, d.g_dst, items, n, d.rope, H, k_mul, v_mul);
     count_launch();
     return cudaGetLastError();
 }
 
 template <bool TO_8BIT>
 cudaError_t launch_dir(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst, bool rotate,
-                       float k_mul, float v_mul, const int32_t *g_src, int first_item, int n, cudaStream_t st) {
+                       float k_mul, float v_mul, const int32_t *g_src, int first_item, int n, int max_blocks, cudaStream_t st) {
     const bool il = pl->cfg.rope_pairing == 1;
     if (pl->cfg.head_dim == 128)
-        return il ? launch_d<128, TO_8BIT, true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, st)
-                  : launch_d<128, TO_8BIT, false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, st);
-    return il ? launch_d<64, TO_8BIT, true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, st)
-              : launch_d<64, TO_8BIT, false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, st);
+        return il ? launch_d<128, TO_8BIT, true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, max_blocks, st)
+                  : launch_d<128, TO_8BIT, false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, max_blocks, st);
+    return il ? launch_d<64, TO_8BIT, true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, max_blocks, st)
+              : launch_d<64, TO_8BIT, false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n, max_blocks, st);
 }
 
 }  // namespace
 
 cudaError_t launch_kv_fp8_range(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst,
                                 bool to_8bit, bool rotate, float k_mul, float v_mul, const int32_t *g_src, int first_item,
-                                int n_items, cudaStream_t st) {
-    return to_8bit ? launch_dir<true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n_items, st)
-                   : launch_dir<false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n_items, st);
+                                int n_items, int max_blocks, cudaStream_t st) {
+    return to_8bit ? launch_dir<true>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n_items, max_blocks, st)
+                   : launch_dir<false>(pl, k_src, v_src, k_dst, v_dst, rotate, k_mul, v_mul, g_src, first_item, n_items, max_blocks, st);
 }
 
 cudaError_t launch_kv_fp8(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst,
                           bool to_8bit, bool rotate, float k_mul, float v_mul, cudaStream_t st) {
     return launch_kv_fp8_range(pl, k_src, v_src, k_dst, v_dst, to_8bit, rotate, k_mul, v_mul, pl->dev.g_src, 0,
-                               (int)pl->items.size(), st);
+                               (int)pl->items.size(), 0, st);
 }
 
 }  // namespace tessera

@@ -14,13 +14,15 @@ void count_launch();   // bumps the process-wide kernel-launch counter
 // separate source pool - and written to the plan's destination slots in (k_pool, v_pool).
 cudaError_t launch_gather(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
                           GatherMode mode, cudaStream_t st);
-// The same kernel over items [first_item, first_item + n_items) of the plan, with the source slots taken
-// from `g_src` (device, indexed like the plan's copy list) instead of the plan's own list.
+// The same kernels over items [first_item, first_item + n_items) of the plan, with the source slots taken
+// from `g_src` (device, indexed like the plan's copy list).  max_blocks > 0 caps the grid: the blocks
+// then walk the items, so the launch occupies only a few SMs (host-tier reader beside the attention kernel).
 cudaError_t launch_gather_range(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool, void *v_pool,
-                                GatherMode mode, const int32_t *g_src, int first_item, int n_items, cudaStream_t st);
+                                GatherMode mode, const int32_t *g_src, int first_item, int n_items, int max_blocks,
+                                cudaStream_t st);
 cudaError_t launch_kv_fp8_range(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst,
                                 bool to_8bit, bool rotate, float k_mul, float v_mul, const int32_t *g_src, int first_item,
-                                int n_items, cudaStream_t st);
+                                int n_items, int max_blocks, cudaStream_t st);
 // 8-bit (e4m3) tier.  to_8bit false: (k_src, v_src) hold codes, (k_dst, v_dst) 16-bit pages, mul = scale;
 // to_8bit true: the reverse, mul = 1 / scale.  Copy list and shift table are the plan's.
 cudaError_t launch_kv_fp8(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst,
@@ -37,7 +39,8 @@ cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_p
                                  const void *v_new, int chunk, cudaStream_t st);
 // tcgen05 attention; returns cudaErrorNotSupported when the plan's shape is outside its range (the plan
 // builder accepts no such shape).
+// max_blocks > 0 caps the persistent grid below one block per SM (SMs left to a concurrent reader kernel).
 cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
-                           float *lse, int chunk, cudaStream_t st, std::string *err);
+                           float *lse, int chunk, int max_blocks, cudaStream_t st, std::string *err);
 
 }  // namespace tessera

@@ -254,7 +254,9 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
         while (item_tokens > 8 && cached / item_tokens < 4 * num_sms) item_tokens /= 2;
     }
     pl->cached_tokens = 0;
-    for (int r = 0; r < batch; ++r)
+    std::vector<int32_t> req_item_off(batch + 1, 0);       // gather items are emitted request by request
+    for (int r = 0; r < batch; ++r) {
+        req_item_off[r] = (int32_t)pl->items.size();
         for (int u = d->unit_off[r]; u < d->unit_off[r + 1]; ++u) {
             if (d->unit_page_off[u + 1] <= d->unit_page_off[u]) continue;
             const int len = d->unit_len[u], tp = d->unit_target_pos[u];
@@ -272,6 +274,8 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
             }
             pl->cached_tokens += len;
         }
+    }
+    req_item_off[batch] = (int32_t)pl->items.size();
 
     // ---- attention work list: tiles of consecutive recompute rows of one request
     const int g = Hq / Hkv;
@@ -386,6 +390,10 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
             pl->chunk_row_off.push_back(n_q);
         }
         const int used_chunks = (int)pl->chunk_row_off.size() - 1;
+        pl->chunk_item_off.assign(used_chunks + 1, (int32_t)pl->items.size());
+        pl->chunk_item_off[0] = 0;
+        for (int r = 1; r < batch; ++r)
+            if (chunk_of[r] != chunk_of[r - 1]) pl->chunk_item_off[chunk_of[r]] = req_item_off[r];
         pl->work_chunked = pl->work;
         std::stable_sort(pl->work_chunked.begin(), pl->work_chunked.end(), [&](const AttnWork &x, const AttnWork &y) {
             return chunk_of[pl->tiles[x.tile_a].req] < chunk_of[pl->tiles[y.tile_a].req];

@@ -98,6 +98,7 @@ struct tessera_plan {
     // The host-buffer entry point pipelines copies against compute over chunks of whole requests.
     std::vector<tessera::AttnWork> work_chunked;   // items of chunk c: [chunk_work_off[c], chunk_work_off[c+1])
     std::vector<int32_t> chunk_work_off, chunk_row_off;   // [n_chunks + 1]; rows = recompute rows
+    std::vector<int32_t> chunk_item_off;                  // [n_chunks + 1]; gather items of the chunk's requests
     std::vector<tessera::CombineItem> combine;     // grouped by chunk: [chunk_combine_off[c], chunk_combine_off[c+1])
     std::vector<int32_t> chunk_combine_off;
     int32_t max_parts = 1;                         // split-KV parts per item (1 = no split)
