@@ -346,6 +346,62 @@ class Leg:
         res["ok"] = bool(res["ok"] and res["kernel_status"] == 0)
         return res, s
 
+    def extend_write_record(self, steps, warmup, peaks):
+        """Write side of the extend pass, two ways, on this leg's workload: un-rotated fresh projections
+        -> (a) tessera_rope_fresh then the attention call's own scatter, (b) the fused tessera_extend_write
+        and attention without scatter.  Times the write kernels alone (L2 flushed) and the whole layer."""
+        import torch
+        t = self.layers[0]
+        sh, n_q = self.w.shape, self.w.n_q
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=self.dev)
+        stream = self.stream
+
+        def timed(fn, do_flush):
+            ms = []
+            for i in range(warmup + steps):
+                if do_flush:
+                    flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                torch.cuda.synchronize()
+                if i >= warmup:
+                    ms.append(a.elapsed_time(b))
+            return sum(ms) / len(ms)
+
+        p = self.plan
+        # a scatter by itself is not an entry point: the unfused write side is timed as the difference
+        # between the attention call with and without its scatter
+        m_rot = timed(lambda: p.rope_fresh(t.q, t.k_new), True)
+        m_att_scatter = timed(lambda: p.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, self.out, self.lse), True)
+        m_att_plain = timed(lambda: p.partial_prefill_attn(t.k_pool, t.v_pool, t.q, None, None, self.out, self.lse), True)
+        m_fused = timed(lambda: p.extend_write(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new), True)
+
+        def layer_unfused():
+            p.kv_compose(t.k_pool, t.v_pool, fuse_rope=True)
+            p.rope_fresh(t.q, t.k_new)
+            p.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, self.out, self.lse)
+
+        def layer_fused():
+            p.kv_compose(t.k_pool, t.v_pool, fuse_rope=True)
+            p.extend_write(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new)
+            p.partial_prefill_attn(t.k_pool, t.v_pool, t.q, None, None, self.out, self.lse)
+
+        m_layer_unfused = timed(layer_unfused, self.flush is not None)
+        m_layer_fused = timed(layer_fused, self.flush is not None)
+        kv_row = sh.num_kv_heads * sh.head_dim * 2
+        q_row = sh.num_q_heads * sh.head_dim * 2
+        fused_bytes = n_q * (2 * q_row + 4 * kv_row)                 # q read + written, K and V read + written once
+        unfused_bytes = n_q * (2 * q_row + 2 * kv_row + 4 * kv_row)  # + the rotated K written in place and read again
+        return {"workload": self.w.name, "recompute_rows": n_q, "steps": steps,
+                "rope_fresh_ms": m_rot, "scatter_ms": m_att_scatter - m_att_plain,
+                "unfused_write_ms": m_rot + m_att_scatter - m_att_plain, "unfused_bytes": int(unfused_bytes),
+                "extend_write_ms": m_fused, "extend_write_bytes": int(fused_bytes),
+                "extend_write_GBps": fused_bytes / m_fused / 1e6,
+                "extend_write_frac_of_measured_copy": fused_bytes / m_fused / 1e6 / peaks["hbm_gbs"],
+                "layer_ms_unfused": m_layer_unfused, "layer_ms_fused": m_layer_fused}
+
     def close(self):
         self.plan.destroy()
         self.layers = None
@@ -750,6 +806,8 @@ def main():
                 par, s = lg.parity(3.0, 2048)
                 rec["parity_ok"], rec["parity"] = par["ok"], par
                 rec["cpu_oracle_tokens_per_s"] = wc.total_tokens / s["layer_seconds_extrapolated"]
+            if c in (3, 5):
+                rec["extend_write"] = lg.extend_write_record(5, 2, peaks)
             per_config.append(rec)
             lg.close()
             del lg

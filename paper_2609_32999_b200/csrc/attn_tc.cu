@@ -72,7 +72,8 @@ struct Barriers {
     uint64_t q_full[2], q_empty[2];
     uint64_t full[kRing], empty[kRing];
     uint64_t s_full[2];
-    uint64_t p_full[2];
+    uint64_t p_half[2][2];     // probabilities of keys [0, 64) / [64, 128) of the tile's current step are in TMEM
+    uint64_t pv_half[2];       // P.V of the first 64 keys has completed (read only when a reference maximum is refreshed mid-step)
     uint64_t pv_done[2];
 };
 
@@ -176,7 +177,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             mbar_init(smem_u32(&bars.q_full[i]), 1);
             mbar_init(smem_u32(&bars.q_empty[i]), 1);
             mbar_init(smem_u32(&bars.s_full[i]), 1);
-            mbar_init(smem_u32(&bars.p_full[i]), 2 * kRows);
+            mbar_init(smem_u32(&bars.p_half[i][0]), 2 * kRows);
+            mbar_init(smem_u32(&bars.p_half[i][1]), 2 * kRows);
+            mbar_init(smem_u32(&bars.pv_half[i]), 1);
             mbar_init(smem_u32(&bars.pv_done[i]), 1);
         }
         for (int i = 0; i < kRing; ++i) {
@@ -356,13 +359,26 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 const bool next_s = j + 1 < my_steps;
                 if (more) ring_wait(2 * j + 2, 3);                     // K_{j+1}
                 const uint32_t vbase = smem_u32(sm + kSmemRing + vslot * kSlotBytes);
-                mbar_wait(smem_u32(&bars.p_full[q]), (step_base + j) & 1, abort_flag, status, 6);
+                // P arrives in two halves: P.V of the first 64 keys runs while the softmax warps are still
+                // on the exponentials of the other 64
+                mbar_wait(smem_u32(&bars.p_half[q][0]), (step_base + j) & 1, abort_flag, status, 6);
                 tc_fence_after();
                 if (lane == 0) {
 #pragma unroll
-                    for (int k = 0; k < kStep / 16; ++k) {
+                    for (int k = 0; k < kStep / 32; ++k) {
                         const uint64_t b = smem_desc_sw128(vbase + k * 2048, kHalfBytes, 1024);
                         umma_ts(tO, tS + k * 8, b, idesc_o, (j > 0) || (k > 0));   // P of keys [16k, 16k + 16): columns 8k .. 8k + 7
+                    }
+                    umma_commit(smem_u32(&bars.pv_half[q]));
+                }
+                __syncwarp();
+                mbar_wait(smem_u32(&bars.p_half[q][1]), (step_base + j) & 1, abort_flag, status, 11);
+                tc_fence_after();
+                if (lane == 0) {
+#pragma unroll
+                    for (int k = kStep / 32; k < kStep / 16; ++k) {
+                        const uint64_t b = smem_desc_sw128(vbase + k * 2048, kHalfBytes, 1024);
+                        umma_ts(tO, tS + k * 8, b, idesc_o, true);
                     }
                     umma_commit(smem_u32(&bars.pv_done[q]));
                     umma_commit(smem_u32(&bars.empty[vslot]));
@@ -437,75 +453,69 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                 const int key0 = (step0 + j) * kStep;
                 const bool masked = key0 + kStep > (q ? t1.kv_full : t0.kv_full);   // a causal limit falls in this step
 
-                uint32_t pk[32];
-                float sum[2] = {0.f, 0.f}, mx[2] = {-INFINITY, -INFINITY};
-                // One pass over this thread's 2 x 32 scores: the row maxima (with_max) and / or the
-                // probabilities against the current reference maxima (with_exp).
-                auto pass = [&](bool with_max, bool with_exp) {
-                    uint32_t s[64];
-                    tmem_ld_16x256b_x16(tS, s);
-                    tmem_wait_ld();
-                    if (masked) {
+                // The thread's 2 x 64 scores (rows t/4 and t/4 + 8 of the warp's 16; of every group of 8
+                // columns, columns 2 (t%4) and 2 (t%4) + 1) stay in registers for the whole step.
+                uint32_t s[64];
+                tmem_ld_16x256b_x16(tS, s);
+                tmem_wait_ld();
+                if (masked) {
 #pragma unroll
-                        for (int k = 0; k < 16; ++k)
+                    for (int k = 0; k < 16; ++k)
 #pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                if (key0 + 8 * k + cq + (e & 1) > p_row[q][e >> 1]) s[4 * k + e] = 0xff800000u;   // -inf
-                    }
-                    if (with_max) {
+                        for (int e = 0; e < 4; ++e)
+                            if (key0 + 8 * k + cq + (e & 1) > p_row[q][e >> 1]) s[4 * k + e] = 0xff800000u;   // -inf
+                }
+                uint32_t pk[16];
+                // Probabilities of column groups [8 h, 8 h + 8) (keys [64 h, 64 h + 64)) against the current
+                // reference maxima: packed into pk, this thread's share of the two row sums into sum.
+                auto exp_half = [&](int h, float (&sum)[2]) {
+                    float sa[2][2] = {{0.f, 0.f}, {0.f, 0.f}}, sb[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+                    // a row that has seen no visible key yet (possible in a later split-KV part) keeps
+                    // the reference at 0: its scores are all -inf and its probabilities 0
+                    const float neg_m[2] = {m_row[q][0] == -INFINITY ? 0.f : -m_row[q][0],
+                                            m_row[q][1] == -INFINITY ? 0.f : -m_row[q][1]};
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
 #pragma unroll
                         for (int rr = 0; rr < 2; ++rr) {
-                            float ma = -INFINITY, mb = -INFINITY;
-#pragma unroll
-                            for (int k = 0; k < 16; ++k) {
-                                ma = fmaxf(ma, __uint_as_float(s[4 * k + 2 * rr]));
-                                mb = fmaxf(mb, __uint_as_float(s[4 * k + 2 * rr + 1]));
-                            }
-                            mx[rr] = quad_max(fmaxf(ma, mb));
+                            const int i = 4 * (8 * h + k) + 2 * rr;
+                            float x0, x1;
+                            fma2(x0, x1, __uint_as_float(s[i]), __uint_as_float(s[i + 1]), scale_log2, neg_m[rr]);
+                            const float e0 = ex2(x0), e1 = ex2(x1);
+                            add2(sa[rr][k & 1], sb[rr][k & 1], e0, e1);
+                            pk[2 * k + rr] = pack_bf16(e0, e1);          // P column 4 (8 h + k) + t%4 of row rr
                         }
-                    }
-                    if (with_exp) {
-                        float sa[2][2] = {{0.f, 0.f}, {0.f, 0.f}}, sb[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-                        // a row that has seen no visible key yet (possible in a later split-KV part) keeps
-                        // the reference at 0: its scores are all -inf and its probabilities 0
-                        const float neg_m[2] = {m_row[q][0] == -INFINITY ? 0.f : -m_row[q][0],
-                                                m_row[q][1] == -INFINITY ? 0.f : -m_row[q][1]};
-#pragma unroll
-                        for (int k = 0; k < 16; ++k)
-#pragma unroll
-                            for (int rr = 0; rr < 2; ++rr) {
-                                float x0, x1;
-                                fma2(x0, x1, __uint_as_float(s[4 * k + 2 * rr]), __uint_as_float(s[4 * k + 2 * rr + 1]), scale_log2, neg_m[rr]);
-                                const float e0 = ex2(x0), e1 = ex2(x1);
-                                add2(sa[rr][k & 1], sb[rr][k & 1], e0, e1);
-                                pk[2 * k + rr] = pack_bf16(e0, e1);      // P column 4k + t%4 of row rr
-                            }
-                        sum[0] = (sa[0][0] + sb[0][0]) + (sa[0][1] + sb[0][1]);
-                        sum[1] = (sa[1][0] + sb[1][0]) + (sa[1][1] + sb[1][1]);
-                    }
+                    sum[0] = (sa[0][0] + sb[0][0]) + (sa[0][1] + sb[0][1]);
+                    sum[1] = (sa[1][0] + sb[1][0]) + (sa[1][1] + sb[1][1]);
                 };
-
-                // Fast path: probabilities against the current reference maxima.  While every thread's
-                // share of a row sum stays below 2^6 the row sum stays below 2^8, every probability
-                // does too and the reference is good enough; otherwise (and on the first step) the
-                // warp's rows take the step's true maxima and redo P.  The decision is per warp.
-                bool stale = true;
-                if (j > 0) {
-                    pass(false, true);
-                    stale = !(sum[0] <= 64.f && sum[1] <= 64.f);
-                }
-                float factor[2] = {1.f, 1.f};
-                if (__any_sync(0xffffffffu, stale)) {
-                    pass(true, false);
+                // P as bf16 over the first 64 columns of S (column c holds keys 2c and 2c + 1), one half at
+                // a time; the MMA warp starts P.V of a half as soon as all 256 threads have stored it.
+                auto release_half = [&](int h) {
+                    tmem_st_16x128b_x8(tS + 32 * h, pk);
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&bars.p_half[q][h]));
+                };
+                // The step's true row maxima become the reference (per warp: all its rows together); the
+                // accumulator and the running sum are brought to the new reference.
+                auto refresh = [&](bool rescale_o, float (&factor)[2]) {
 #pragma unroll
                     for (int rr = 0; rr < 2; ++rr) {
-                        const float mc = fmaxf(m_row[q][rr], mx[rr] * scale_log2);
+                        float ma = -INFINITY, mb = -INFINITY;
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            ma = fmaxf(ma, __uint_as_float(s[4 * k + 2 * rr]));
+                            mb = fmaxf(mb, __uint_as_float(s[4 * k + 2 * rr + 1]));
+                        }
+                        const float mx = quad_max(fmaxf(ma, mb));
+                        const float mc = fmaxf(m_row[q][rr], mx * scale_log2);
+                        factor[rr] = 1.f;
                         if (mc != -INFINITY) {
                             factor[rr] = ex2(m_row[q][rr] - mc);   // 0 when the row had no visible key before
                             m_row[q][rr] = mc;
                         }
                     }
-                    if (j > 0) {
+                    if (rescale_o) {
                         const uint32_t tO = tmem + kTmemO + q * 128 + lane_base;
                         uint32_t o[kD / 2];
                         if constexpr (kD == 128) tmem_ld_16x256b_x16(tO, o); else tmem_ld_16x256b_x8(tO, o);
@@ -514,15 +524,42 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                         for (int i = 0; i < kD / 2; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor[(i >> 1) & 1]);
                         if constexpr (kD == 128) tmem_st_16x256b_x16(tO, o); else tmem_st_16x256b_x8(tO, o);
                     }
-                    pass(false, true);
+                };
+
+                // Fast path: probabilities against the current reference maxima.  While every thread's
+                // share of a row sum stays below 2^6 the row sum stays below 2^8, every probability
+                // does too and the reference is good enough; otherwise (and on the first step) the
+                // warp's rows take the step's true maxima.  The decision is per warp, and it is taken
+                // after each half: once the first half has been released, a refresh concerns only the
+                // second half (the first half's P.V is brought to the new reference with the accumulator).
+                float sum_a[2], sum_b[2], factor[2];
+                bool fresh = j == 0;
+                if (!fresh) {
+                    exp_half(0, sum_a);
+                    fresh = __any_sync(0xffffffffu, !(sum_a[0] <= 64.f && sum_a[1] <= 64.f));
                 }
-                l_row[q][0] = l_row[q][0] * factor[0] + sum[0];
-                l_row[q][1] = l_row[q][1] * factor[1] + sum[1];
-                // P as bf16 over the first 64 columns of S: column c holds keys 2c and 2c + 1
-                tmem_st_16x128b_x16(tS, pk);
-                tmem_wait_st();
-                tc_fence_before();
-                mbar_arrive(smem_u32(&bars.p_full[q]));
+                if (fresh) {
+                    refresh(j > 0, factor);       // S_j complete means P.V of step j - 1 has completed: O is at rest
+                    exp_half(0, sum_a);
+                    l_row[q][0] *= factor[0];
+                    l_row[q][1] *= factor[1];
+                }
+                release_half(0);
+                exp_half(1, sum_b);
+                if (!fresh && __any_sync(0xffffffffu, !(sum_a[0] + sum_b[0] <= 64.f && sum_a[1] + sum_b[1] <= 64.f))) {
+                    // the first half is already with the MMA warp, in units of the old reference: wait until
+                    // its P.V has landed in the accumulator, then move accumulator and sums to the new one
+                    mbar_wait(smem_u32(&bars.pv_half[q]), par, abort_flag, status, 12);
+                    tc_fence_after();
+                    refresh(true, factor);
+                    l_row[q][0] = (l_row[q][0] + sum_a[0]) * factor[0];
+                    l_row[q][1] = (l_row[q][1] + sum_a[1]) * factor[1];
+                    sum_a[0] = sum_a[1] = 0.f;
+                    exp_half(1, sum_b);
+                }
+                l_row[q][0] += sum_a[0] + sum_b[0];
+                l_row[q][1] += sum_a[1] + sum_b[1];
+                release_half(1);
             }
         }
 
