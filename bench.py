@@ -349,7 +349,8 @@ class Leg:
     def extend_write_record(self, steps, warmup, peaks):
         """Write side of the extend pass, two ways, on this leg's workload: un-rotated fresh projections
         -> (a) tessera_rope_fresh then the attention call's own scatter, (b) the fused tessera_extend_write
-        and attention without scatter.  Times the write kernels alone (L2 flushed) and the whole layer."""
+        and attention without scatter.  Times the rotation / fused write kernels alone (L2 flushed) and the
+        whole layer both ways."""
         import torch
         t = self.layers[0]
         sh, n_q = self.w.shape, self.w.n_q
@@ -371,11 +372,9 @@ class Leg:
             return sum(ms) / len(ms)
 
         p = self.plan
-        # a scatter by itself is not an entry point: the unfused write side is timed as the difference
-        # between the attention call with and without its scatter
+        # (the scatter of the unfused way is part of the attention call and has no entry point of its own:
+        # its cost shows in the whole-layer times)
         m_rot = timed(lambda: p.rope_fresh(t.q, t.k_new), True)
-        m_att_scatter = timed(lambda: p.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, self.out, self.lse), True)
-        m_att_plain = timed(lambda: p.partial_prefill_attn(t.k_pool, t.v_pool, t.q, None, None, self.out, self.lse), True)
         m_fused = timed(lambda: p.extend_write(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new), True)
 
         def layer_unfused():
@@ -395,8 +394,7 @@ class Leg:
         fused_bytes = n_q * (2 * q_row + 4 * kv_row)                 # q read + written, K and V read + written once
         unfused_bytes = n_q * (2 * q_row + 2 * kv_row + 4 * kv_row)  # + the rotated K written in place and read again
         return {"workload": self.w.name, "recompute_rows": n_q, "steps": steps,
-                "rope_fresh_ms": m_rot, "scatter_ms": m_att_scatter - m_att_plain,
-                "unfused_write_ms": m_rot + m_att_scatter - m_att_plain, "unfused_bytes": int(unfused_bytes),
+                "rope_fresh_ms": m_rot, "unfused_bytes": int(unfused_bytes),
                 "extend_write_ms": m_fused, "extend_write_bytes": int(fused_bytes),
                 "extend_write_GBps": fused_bytes / m_fused / 1e6,
                 "extend_write_frac_of_measured_copy": fused_bytes / m_fused / 1e6 / peaks["hbm_gbs"],
