@@ -171,3 +171,26 @@ def test_capture_descriptor_validation_and_row_count():
     assert tb.plan_create_status(with_capture([0, 0, 2], [int(w0.free_pages[0]), spare[0]])) == tb.PAGE_OUT_OF_RANGE   # a destination page
     assert tb.plan_create_status(with_capture([0, 0, 2], [spare[0], spare[0]])) == tb.PAGE_OUT_OF_RANGE                # listed twice
     assert tb.plan_create_status(with_capture([0, 0, 2], [0, 2], pool=2)) == tb.PAGE_OUT_OF_RANGE                      # outside the cache pool
+
+
+def test_llama31_scaled_frequencies_match_the_library_rule():
+    """The helper's table against the model library's own Llama-3 frequency initialisation."""
+    import torch
+    from transformers import LlamaConfig
+    from transformers.modeling_rope_utils import ROPE_INIT_FUNCTIONS
+    from paper_2609_32999_b200 import rope_scaling as rs
+    scaling = {"rope_type": "llama3", "factor": 8.0, "low_freq_factor": 1.0, "high_freq_factor": 4.0,
+               "original_max_position_embeddings": 8192, "rope_theta": 500000.0}
+    try:
+        cfg = LlamaConfig(hidden_size=4096, num_attention_heads=32, rope_theta=500000.0, max_position_embeddings=131072,
+                          rope_scaling=dict(scaling))
+    except TypeError:
+        cfg = LlamaConfig(hidden_size=4096, num_attention_heads=32, max_position_embeddings=131072, rope_parameters=dict(scaling))
+    want, _ = ROPE_INIT_FUNCTIONS["llama3"](cfg, "cpu")
+    got = rs.llama31_inv_freq(128, 500000.0)
+    assert np.allclose(got, want.double().numpy(), rtol=1e-6)
+    plain = rs.default_inv_freq(128, 500000.0)
+    assert np.array_equal(got[:20], plain[:20]) and np.allclose(got[-10:], plain[-10:] / 8.0)      # fast pairs kept, slow pairs 8x slower
+    # and a plan takes the table
+    w = wl.config(2)
+    assert tb.Plan(w, host_only=True, inv_freq=got).info.n_rope_rows == 10
