@@ -400,6 +400,39 @@ class Leg:
                 "extend_write_frac_of_measured_copy": fused_bytes / m_fused / 1e6 / peaks["hbm_gbs"],
                 "layer_ms_unfused": m_layer_unfused, "layer_ms_fused": m_layer_fused}
 
+    def k8_attention_record(self, steps, warmup, peaks):
+        """Attention over 8-bit key pages (tessera_partial_prefill_attn_k8: queries quantised by the call, fresh
+        rows scattered as codes) against the 16-bit call on the same composed layer; flops are the same
+        algorithmic count (the 8-bit S = Q K^T runs at twice the tensor rate, P.V stays 16-bit)."""
+        import torch
+        t = self.layers[0]
+        p = self.plan
+        p.kv_compose(t.k_pool, t.v_pool, fuse_rope=True)
+        ks = qs = 1.0 / 32
+        k8 = (t.k_pool.float() * (1.0 / ks)).clamp_(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=self.dev)
+        stream = self.stream
+
+        def timed(fn):
+            ms = []
+            for i in range(warmup + steps):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                torch.cuda.synchronize()
+                if i >= warmup:
+                    ms.append(a.elapsed_time(b))
+            return sum(ms) / len(ms)
+
+        m16 = timed(lambda: p.partial_prefill_attn(t.k_pool, t.v_pool, t.q, t.k_new, t.v_new, self.out, self.lse))
+        m8 = timed(lambda: p.partial_prefill_attn_k8(k8, ks, t.v_pool, t.q, qs, t.k_new, t.v_new, self.out, self.lse))
+        flops = p.info.attn_flops
+        return {"workload": self.w.name, "steps": steps, "l2": "flushed between calls",
+                "bf16_ms": m16, "bf16_tflops": flops / m16 / 1e9, "k8_ms": m8, "k8_tflops_algorithmic": flops / m8 / 1e9,
+                "speedup": m16 / m8, "note": "k8 time includes quantising q (one pass over q) and the 8-bit fresh-row scatter"}
+
     def close(self):
         self.plan.destroy()
         self.layers = None
@@ -765,6 +798,9 @@ def main():
     }
     if sustained:
         line["sustained"] = sustained
+    k8_record = None
+    if not args.only_headline and world == 1 and sh.head_dim == 128:
+        k8_record = leg.k8_attention_record(8, 3, peaks)
     if not args.no_cpu_baseline:
         par, s = leg.parity(args.cpu_budget, None)
         line["cpu_baseline"] = {"value": w.total_tokens / s["layer_seconds_extrapolated"], "unit": UNIT,
@@ -815,6 +851,8 @@ def main():
         line["host_tier"] = [host_tier_record(w4, dev, 3, 2), host_tier_record(rank_workload(3, rank, None, None), dev, 5, 2)]
         torch.cuda.empty_cache()
         line["fp8_tier"] = fp8_tier_record(w4, dev, 8, 3, peaks)
+        if k8_record:
+            line["fp8_key_attention"] = k8_record
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

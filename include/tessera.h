@@ -291,6 +291,29 @@ TESSERA_API int32_t tessera_partial_prefill_attn(const tessera_plan *plan, void 
                                      void *out, float *lse, void *stream);
 
 /*
+ * Partial-prefill attention over 8-BIT KEY PAGES.  The paper stores and attends over 16-bit K/V
+ * (Sec. 8, "Algorithm and Model Compatibility") and has no counterpart of this call; it is the extend
+ * pass of Sec. 5.3 as a different numerical method: queries and keys are e4m3 codes (1-4-3 float, largest
+ * value 448), S = Q K^T runs on the 8-bit tensor-core path, probabilities, values and the accumulator stay
+ * as in tessera_partial_prefill_attn.
+ *   k_pool8   device [num_pool_pages][page_size][H_kv][D] bytes: code c stands for c * k_scale.  The
+ *             request's destination pages must hold its assembled keys as codes (e.g. written by
+ *             tessera_kv_retain_fp8 with a compose plan, which rotates and quantises on the way).
+ *   v_pool    device, 16-bit pool as everywhere else
+ *   q         device [n_q][H_q][D] bf16, already rotated; quantised by the call itself into a buffer the
+ *             plan owns (allocated on the first call): code = e4m3_rne(q * fp32(1 / q_scale)), saturating
+ *   k_new, v_new  fresh rows (nullable together): k_new is written to the rows' slots of k_pool8 as
+ *             e4m3_rne(k_new * fp32(1 / k_scale)), v_new to v_pool as bit copies
+ *   out, lse  as in tessera_partial_prefill_attn: out[j][h] = softmax(sm_scale * (q8 q_scale) . (k8 k_scale)) . V
+ * head_dim 128 only (TESSERA_UNSUPPORTED_SHAPE otherwise).  The result is compared with fp64 attention
+ * over the DECODED operands (the codes times their scales) at the usual tolerance: the quantisation is
+ * part of the method, not an error of the kernel.
+ */
+TESSERA_API int32_t tessera_partial_prefill_attn_k8(tessera_plan *plan, void *k_pool8, float k_scale, void *v_pool,
+                                                    const void *q, float q_scale, const void *k_new, const void *v_new,
+                                                    void *out, float *lse, void *stream);
+
+/*
  * The whole per-layer path for callers whose activations live in HOST memory: copies q, k_new,
  * v_new (host, pinned for full speed) to staging buffers owned by the plan, runs fused compose and
  * attention, copies out (and lse when non-null) back to the host and waits for `stream`.

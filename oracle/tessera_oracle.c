@@ -325,41 +325,64 @@ int oracle_assemble_ex(int r, const int32_t *seq_len, const int32_t *unit_off,
  *     O   = sum_t softmax(s)_t V[t]
  *     LSE = log sum_t exp(s_t)
  * ------------------------------------------------------------------------- */
+static void attention_row(const double *qd, int p, int kvh, int H_kv, int D, double scale,
+                          const double *k_asm, const uint16_t *v_asm, double *o, double *lse)
+{
+    size_t row = (size_t)H_kv * D;
+    double *s = (double *)malloc(sizeof(double) * ((size_t)p + 1));
+    double mx = -INFINITY;
+    for (int t = 0; t <= p; ++t) {
+        const double *kv = k_asm + (size_t)t * row + (size_t)kvh * D;
+        double acc = 0.0;
+        for (int d = 0; d < D; ++d) acc += qd[d] * kv[d];
+        s[t] = acc * scale;
+        if (s[t] > mx) mx = s[t];
+    }
+    double denom = 0.0;
+    for (int t = 0; t <= p; ++t) { s[t] = exp(s[t] - mx); denom += s[t]; }
+    for (int d = 0; d < D; ++d) o[d] = 0.0;
+    for (int t = 0; t <= p; ++t) {
+        const uint16_t *vv = v_asm + (size_t)t * row + (size_t)kvh * D;
+        double w = s[t] / denom;
+        for (int d = 0; d < D; ++d) o[d] += w * bf16_to_double(vv[d]);
+    }
+    *lse = mx + log(denom);
+    free(s);
+}
+
 void oracle_attention_rows(int T, int H_q, int H_kv, int D, double scale,
                            const double *k_asm, const uint16_t *v_asm, const uint16_t *q,
                            int n_rows, const int32_t *row_q, const int32_t *row_h, const int32_t *row_pos,
                            double *out, double *lse)
 {
     int g = H_q / H_kv;
-    size_t row = (size_t)H_kv * D;
     (void)T;
 #pragma omp parallel for schedule(dynamic, 4)
     for (int i = 0; i < n_rows; ++i) {
-        int h = row_h[i], kvh = h / g, p = row_pos[i];
+        int h = row_h[i];
         const uint16_t *qv = q + ((size_t)row_q[i] * H_q + h) * D;
         double *qd = (double *)malloc(sizeof(double) * D);
-        double *s = (double *)malloc(sizeof(double) * ((size_t)p + 1));
         for (int d = 0; d < D; ++d) qd[d] = bf16_to_double(qv[d]);
-        double mx = -INFINITY;
-        for (int t = 0; t <= p; ++t) {
-            const double *kv = k_asm + (size_t)t * row + (size_t)kvh * D;
-            double acc = 0.0;
-            for (int d = 0; d < D; ++d) acc += qd[d] * kv[d];
-            s[t] = acc * scale;
-            if (s[t] > mx) mx = s[t];
-        }
-        double denom = 0.0;
-        for (int t = 0; t <= p; ++t) { s[t] = exp(s[t] - mx); denom += s[t]; }
-        double *o = out + (size_t)i * D;
-        for (int d = 0; d < D; ++d) o[d] = 0.0;
-        for (int t = 0; t <= p; ++t) {
-            const uint16_t *vv = v_asm + (size_t)t * row + (size_t)kvh * D;
-            double w = s[t] / denom;
-            for (int d = 0; d < D; ++d) o[d] += w * bf16_to_double(vv[d]);
-        }
-        lse[i] = mx + log(denom);
+        attention_row(qd, row_pos[i], h / g, H_kv, D, scale, k_asm, v_asm, out + (size_t)i * D, lse + i);
         free(qd);
-        free(s);
+    }
+}
+
+/* The same rows with the queries given as doubles [n_q][H_q][D] (queries that are not bf16 numbers: the
+ * decoded values of 8-bit codes times a scale - this build's 8-bit-key attention, which the paper does
+ * not have). */
+void oracle_attention_rows_qf64(int T, int H_q, int H_kv, int D, double scale,
+                                const double *k_asm, const uint16_t *v_asm, const double *q,
+                                int n_rows, const int32_t *row_q, const int32_t *row_h, const int32_t *row_pos,
+                                double *out, double *lse)
+{
+    int g = H_q / H_kv;
+    (void)T;
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int i = 0; i < n_rows; ++i) {
+        int h = row_h[i];
+        attention_row(q + ((size_t)row_q[i] * H_q + h) * D, row_pos[i], h / g, H_kv, D, scale, k_asm, v_asm,
+                      out + (size_t)i * D, lse + i);
     }
 }
 

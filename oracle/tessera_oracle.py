@@ -173,7 +173,8 @@ def attention_rows(w, k_asm: np.ndarray, v_bits: np.ndarray, q_bits: np.ndarray,
                    row_q: Sequence[int], row_h: Sequence[int], row_pos: Sequence[int],
                    scale: Optional[float] = None):
     """O [n_rows, D] (fp64) and LSE [n_rows] for the listed (query token, head) rows
-    of ONE request whose assembled K (fp64) / V (bits) are given."""
+    of ONE request whose assembled K (fp64) / V (bits) are given.  q_bits: bf16 bits (uint16), or the
+    queries themselves as float64 (values that are not bf16 numbers)."""
     sh = w.shape
     if scale is None:
         scale = sh.sm_scale if sh.sm_scale else 1.0 / np.sqrt(sh.head_dim)
@@ -183,10 +184,14 @@ def attention_rows(w, k_asm: np.ndarray, v_bits: np.ndarray, q_bits: np.ndarray,
     lse = np.zeros(n, np.float64)
     k_asm = np.ascontiguousarray(k_asm, dtype=np.float64)
     v_bits = np.ascontiguousarray(v_bits, dtype=np.uint16)
-    lib().oracle_attention_rows(
-        ctypes.c_int(k_asm.shape[0]), ctypes.c_int(sh.num_q_heads), ctypes.c_int(sh.num_kv_heads),
-        ctypes.c_int(sh.head_dim), ctypes.c_double(scale), _p(k_asm), _p(v_bits), _p(q_bits),
-        ctypes.c_int(n), _p(row_q), _p(row_h), _p(row_pos), _p(out), _p(lse))
+    if q_bits.dtype == np.float64:
+        fn, q_arg = lib().oracle_attention_rows_qf64, np.ascontiguousarray(q_bits)
+        fn.restype = None
+    else:
+        fn, q_arg = lib().oracle_attention_rows, q_bits
+    fn(ctypes.c_int(k_asm.shape[0]), ctypes.c_int(sh.num_q_heads), ctypes.c_int(sh.num_kv_heads),
+       ctypes.c_int(sh.head_dim), ctypes.c_double(scale), _p(k_asm), _p(v_bits), _p(q_arg),
+       ctypes.c_int(n), _p(row_q), _p(row_h), _p(row_pos), _p(out), _p(lse))
     return out, lse
 
 

@@ -55,7 +55,7 @@ class PlanInfo(ctypes.Structure):
 
 
 EXPORTS = ["tessera_plan_create", "tessera_plan_destroy", "tessera_plan_block_table", "tessera_plan_get_info",
-           "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_kv_compose_from_fp8", "tessera_kv_retain_fp8", "tessera_rope_shift", "tessera_rope_fresh", "tessera_extend_write", "tessera_partial_prefill_attn",
+           "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_kv_compose_from_fp8", "tessera_kv_retain_fp8", "tessera_rope_shift", "tessera_rope_fresh", "tessera_extend_write", "tessera_partial_prefill_attn", "tessera_partial_prefill_attn_k8",
            "tessera_composed_prefill_host", "tessera_composed_prefill_host_tier", "tessera_rope_shift_static", "tessera_selftest_bounded_wait", "tessera_last_error",
            "tessera_launch_count"]
 
@@ -74,6 +74,7 @@ _lib.tessera_rope_shift.argtypes = [_vp, _vp, _vp]
 _lib.tessera_rope_fresh.argtypes = [_vp, _vp, _vp, _vp]
 _lib.tessera_extend_write.argtypes = [_vp] * 9
 _lib.tessera_partial_prefill_attn.argtypes = [_vp] * 9
+_lib.tessera_partial_prefill_attn_k8.argtypes = [_vp, _vp, ctypes.c_float, _vp, _vp, ctypes.c_float, _vp, _vp, _vp, _vp, _vp]
 _lib.tessera_composed_prefill_host.argtypes = [_vp] * 9
 _lib.tessera_composed_prefill_host_tier.argtypes = [_vp, _vp, _vp, ctypes.c_int32, ctypes.c_float, ctypes.c_float,
                                                     _vp, _vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_int32, _vp]
@@ -218,6 +219,13 @@ class Plan:
     def partial_prefill_attn(self, k_pool, v_pool, q, k_new, v_new, out, lse=None, stream=None) -> None:
         _check(_lib.tessera_partial_prefill_attn(self._h, _dev(k_pool), _dev(v_pool), _dev(q), _dev(k_new),
                                                  _dev(v_new), _dev(out), _dev(lse), _stream(stream)))
+
+    def partial_prefill_attn_k8(self, k_pool8, k_scale: float, v_pool, q, q_scale: float, k_new, v_new, out, lse=None,
+                                stream=None) -> None:
+        """Attention over 8-bit (e4m3) key pages: q is quantised by the call, k_pool8 holds codes."""
+        _check(_lib.tessera_partial_prefill_attn_k8(self._h, _dev(k_pool8), float(k_scale), _dev(v_pool), _dev(q),
+                                                    float(q_scale), _dev(k_new), _dev(v_new), _dev(out), _dev(lse),
+                                                    _stream(stream)))
 
     def composed_prefill_host(self, k_pool, v_pool, q_host, k_new_host, v_new_host, out_host, lse_host=None,
                               stream=None) -> None:

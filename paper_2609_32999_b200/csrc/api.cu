@@ -229,7 +229,7 @@ int32_t tessera_plan_destroy(tessera_plan *pl) {
         if (pl->ev_out) cudaEventDestroy(pl->ev_out);
         if (pl->s_in) cudaStreamDestroy(pl->s_in);
         if (pl->s_out) cudaStreamDestroy(pl->s_out);
-        void *bufs[] = {pl->dev.blob, pl->dev.st_q, pl->dev.st_k, pl->dev.st_v, pl->dev.st_o, pl->dev.st_lse};
+        void *bufs[] = {pl->dev.blob, pl->dev.st_q, pl->dev.st_k, pl->dev.st_v, pl->dev.st_o, pl->dev.st_lse, pl->dev.q8};
         for (void *b : bufs)
             if (b) {
                 cudaError_t e = cudaFree(b);
@@ -375,6 +375,31 @@ int32_t tessera_partial_prefill_attn(const tessera_plan *pl, void *k_pool, void 
     if (misaligned(q) || misaligned(out) || misaligned(k_new) || misaligned(v_new))
         return set_error(TESSERA_INVALID_ARG, "q / out / k_new / v_new must be 16-byte aligned");
     return attention(pl, k_pool, v_pool, q, k_new, v_new, out, lse, -1, static_cast<cudaStream_t>(stream));
+}
+
+int32_t tessera_partial_prefill_attn_k8(tessera_plan *pl, void *k_pool8, float k_scale, void *v_pool, const void *q,
+                                        float q_scale, const void *k_new, const void *v_new, void *out, float *lse,
+                                        void *stream) {
+    if (int32_t rc = check_device_plan(pl)) return rc;
+    if (pl->cfg.head_dim != 128) return set_error(TESSERA_UNSUPPORTED_SHAPE, "8-bit keys: head_dim 128 only");
+    if (!k_pool8 || !v_pool || misaligned(k_pool8) || misaligned(v_pool))
+        return set_error(TESSERA_INVALID_ARG, "k_pool8 / v_pool must be non-null and 16-byte aligned");
+    if (!(k_scale > 0.f) || !(q_scale > 0.f) || std::isinf(k_scale) || std::isinf(q_scale))
+        return set_error(TESSERA_INVALID_ARG, "k_scale / q_scale must be positive and finite");
+    if (pl->n_q > 0 && (!q || !out)) return set_error(TESSERA_INVALID_ARG, "q and out must be non-null");
+    if (misaligned(q) || misaligned(out) || misaligned(k_new) || misaligned(v_new))
+        return set_error(TESSERA_INVALID_ARG, "q / out / k_new / v_new must be 16-byte aligned");
+    if (pl->n_q == 0) return TESSERA_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t q_elems = pl->n_q * pl->cfg.num_q_heads * pl->cfg.head_dim;
+    if (!pl->dev.q8) TS_CUDA(cudaMalloc(&pl->dev.q8, (size_t)q_elems));
+    // the reciprocals are taken once, in fp32: every element is multiplied by it and rounded to e4m3
+    TS_CUDA(launch_quantize_e4m3(q, pl->dev.q8, q_elems, 1.0f / q_scale, st));
+    TS_CUDA(launch_scatter_fresh_k8(pl, k_pool8, v_pool, k_new, v_new, 1.0f / k_scale, st));
+    std::string err;
+    cudaError_t e = launch_attn_tc_k8(pl, k_pool8, v_pool, pl->dev.q8, out, lse, q_scale * k_scale, st, &err);
+    if (e != cudaSuccess) return set_error(TESSERA_CUDA_ERROR, "tcgen05 attention launch (8-bit keys): " + err + " / " + cudaGetErrorString(e));
+    return TESSERA_OK;
 }
 
 int32_t tessera_composed_prefill_host(tessera_plan *pl, void *k_pool, void *v_pool, const void *q_host,

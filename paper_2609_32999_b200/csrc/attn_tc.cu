@@ -114,7 +114,10 @@ struct Item {
 
 // kMaxPages: most pages a 128-key step can consist of in this instantiation - 8 (pages of 16 tokens or
 // more) or 16 (pages of 8 tokens); the wider producer loop is kept out of the common instantiation.
-template <int D, int kMaxPages>
+// K8: queries and keys are 8-bit floats (e4m3 codes; the scales are folded into scale_log2 by the host):
+// S = Q K^T runs as kind::f8f6f4 with 32 elements of head_dim per instruction, a Q tile and a K step are
+// 128 rows of 128 bytes (one swizzle atom wide, head_dim 128 only); V, P and the accumulator stay as they are.
+template <int D, int kMaxPages, bool K8>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
@@ -129,6 +132,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     using G = Geo<D>;
     constexpr int kD = D;
     constexpr uint32_t kQTileBytes = G::kQTileBytes, kSlotBytes = G::kSlotBytes;
+    constexpr int kQKHalves = K8 ? 1 : G::kHalves;      // 128-byte-wide halves of a Q tile / a K step
     constexpr uint32_t kSmemQ = G::kSmemQ, kSmemRing = G::kSmemRing;
     __shared__ __align__(8) Barriers bars;
     __shared__ uint32_t s_tmem_base;
@@ -217,7 +221,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         if (q_rows < kRows) {
             for (int q = 0; q < 2; ++q)
 #pragma unroll
-                for (int hf = 0; hf < G::kHalves; ++hf) {
+                for (int hf = 0; hf < kQKHalves; ++hf) {
                     uint8_t *base = sm + kSmemQ + q * kQTileBytes + hf * kHalfBytes;
                     for (int o = q_rows * 128 + lane * 16; o < kRows * 128; o += 32 * 16)
                         *reinterpret_cast<uint4 *>(base + o) = make_uint4(0, 0, 0, 0);
@@ -240,9 +244,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                     // the previous item's last S MMA has read this buffer
                     if (q_uses[q] > 0) mbar_wait(smem_u32(&bars.q_empty[q]), (q_uses[q] - 1) & 1, abort_flag, status, 10);
                     const uint32_t bar = smem_u32(&bars.q_full[q]);
-                    mbar_expect_tx(bar, (uint32_t)(G::kHalves * q_rows * 128));
+                    mbar_expect_tx(bar, (uint32_t)(kQKHalves * q_rows * 128));
 #pragma unroll
-                    for (int hf = 0; hf < G::kHalves; ++hf)
+                    for (int hf = 0; hf < kQKHalves; ++hf)
                         tma_load_3d(smem_u32(sm + kSmemQ + q * kQTileBytes + hf * kHalfBytes), &tmap_q, bar, hf * 64, kvh * g, t.q_begin);
                 }
             }
@@ -265,7 +269,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                             const int item = ring_base + 2 * j + kv, slot = item % kRing;
                             mbar_wait(smem_u32(&bars.empty[slot]), ((item / kRing) & 1) ^ 1, abort_flag, status, 1 + kv);
                             const uint32_t fb = smem_u32(&bars.full[slot]);
-                            mbar_expect_tx(fb, kSlotBytes);
+                            const int halves = kv ? G::kHalves : kQKHalves;
+                            mbar_expect_tx(fb, (uint32_t)halves * kHalfBytes);
                             const uint32_t dst = smem_u32(sm + kSmemRing + slot * kSlotBytes);
                             const CUtensorMap *tm = kv ? &tmap_v : &tmap_k;
 #pragma unroll
@@ -273,7 +278,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                                 if (k < pps) {
 #pragma unroll
                                     for (int hf = 0; hf < G::kHalves; ++hf)
-                                        tma_load_4d(dst + hf * kHalfBytes + k * page_bytes, tm, fb, hf * 64, kvh, 0, pg[k]);
+                                        if (hf < halves) tma_load_4d(dst + hf * kHalfBytes + k * page_bytes, tm, fb, hf * 64, kvh, 0, pg[k]);
                                 }
                         }
                     }
@@ -287,7 +292,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         // tile 0, warp 10 for tile 1.  Each runs its own tile's chain, so the waits of one overlap
         // the MMAs of the other; a ring slot is free again once both have released it (the warp of a
         // tile that is absent or already finished only releases).
-        constexpr uint32_t idesc_s = idesc_bf16(kRows, kStep, false);
+        constexpr uint32_t idesc_s = K8 ? idesc_e4m3(kRows, kStep) : idesc_bf16(kRows, kStep, false);
         constexpr uint32_t idesc_o = idesc_bf16(kRows, kD, true);
         const int q = warp - 9;
         const uint32_t qbase = smem_u32(sm + kSmemQ + q * kQTileBytes);
@@ -311,11 +316,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             auto slot_of = [&](int item) { return (ring_base + item) % kRing; };
             auto issue_s = [&](int j) {                                // S[q] = Q_q K_j^T (lane 0)
                 const uint32_t kbase = smem_u32(sm + kSmemRing + slot_of(2 * j) * kSlotBytes);
+                if constexpr (K8) {
 #pragma unroll
-                for (int k = 0; k < kD / 16; ++k) {
-                    const uint64_t a = smem_desc_sw128(qbase + (k / 4) * kHalfBytes + (k % 4) * 32, 16, 1024);
-                    const uint64_t b = smem_desc_sw128(kbase + (k / 4) * kHalfBytes + (k % 4) * 32, 16, 1024);
-                    umma_ss(tS, a, b, idesc_s, k > 0);
+                    for (int k = 0; k < kD / 32; ++k) {                // 32 bytes = 32 elements of head_dim per instruction
+                        const uint64_t a = smem_desc_sw128(qbase + k * 32, 16, 1024);
+                        const uint64_t b = smem_desc_sw128(kbase + k * 32, 16, 1024);
+                        umma_ss_f8(tS, a, b, idesc_s, k > 0);
+                    }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < kD / 16; ++k) {
+                        const uint64_t a = smem_desc_sw128(qbase + (k / 4) * kHalfBytes + (k % 4) * 32, 16, 1024);
+                        const uint64_t b = smem_desc_sw128(kbase + (k / 4) * kHalfBytes + (k % 4) * 32, 16, 1024);
+                        umma_ss(tS, a, b, idesc_s, k > 0);
+                    }
                 }
                 umma_commit(smem_u32(&bars.s_full[q]));
                 umma_commit(smem_u32(&bars.empty[slot_of(2 * j)]));    // K_j no longer needed by this tile
@@ -701,28 +715,33 @@ attn_combine_kernel(const CombineItem *__restrict__ items, const AttnTile *__res
     if (lse && lane == 0) lse[(size_t)tok * H_q + head] = (m + log2f(l)) * 0.6931471805599453f;
 }
 
-template <int D, int kMaxPages>
+template <int D, int kMaxPages, bool K8>
 cudaError_t launch_attn_tc_d(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
-                             float *lse, int chunk, int max_blocks, cudaStream_t st, std::string *err) {
+                             float *lse, int chunk, int max_blocks, float qk_scale, cudaStream_t st, std::string *err) {
     const AttnWork *work = chunk < 0 ? pl->dev.work : pl->dev.work_chunked + pl->chunk_work_off[chunk];
     const size_t n_work = chunk < 0 ? pl->work.size() : (size_t)(pl->chunk_work_off[chunk + 1] - pl->chunk_work_off[chunk]);
     if (n_work == 0) return cudaSuccess;
     const int Hq = pl->cfg.num_q_heads, Hkv = pl->cfg.num_kv_heads, g = Hq / Hkv, ps = pl->cfg.page_size;
     CUtensorMap tq, tk, tv, to;
-    if (!make_q_tmap(&tq, q, pl->n_q, Hq, D, g, kRows / g, err)) return cudaErrorInvalidValue;
-    if (!make_q_tmap(&to, out, pl->n_q, Hq, D, g, kRows / g, err)) return cudaErrorInvalidValue;   // `out` has the layout of q
-    if (!make_pool_tmap(&tk, k_pool, pl->num_pool_pages, ps, Hkv, D, err)) return cudaErrorInvalidValue;
+    if (K8) {      // q and k_pool hold one byte per element
+        if (!make_q_tmap8(&tq, q, pl->n_q, Hq, D, g, kRows / g, err)) return cudaErrorInvalidValue;
+        if (!make_pool_tmap8(&tk, k_pool, pl->num_pool_pages, ps, Hkv, D, err)) return cudaErrorInvalidValue;
+    } else {
+        if (!make_q_tmap(&tq, q, pl->n_q, Hq, D, g, kRows / g, err)) return cudaErrorInvalidValue;
+        if (!make_pool_tmap(&tk, k_pool, pl->num_pool_pages, ps, Hkv, D, err)) return cudaErrorInvalidValue;
+    }
+    if (!make_q_tmap(&to, out, pl->n_q, Hq, D, g, kRows / g, err)) return cudaErrorInvalidValue;   // `out` has the layout of a 16-bit q
     if (!make_pool_tmap(&tv, v_pool, pl->num_pool_pages, ps, Hkv, D, err)) return cudaErrorInvalidValue;
     {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D, kMaxPages>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Geo<D>::kSmemAlloc);
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D, kMaxPages, K8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Geo<D>::kSmemAlloc);
         if (e != cudaSuccess) { *err = "cudaFuncSetAttribute(shared memory)"; return e; }
     }
     const DeviceTables &d = pl->dev;
-    const float scale_log2 = pl->sm_scale * 1.4426950408889634f;
+    const float scale_log2 = pl->sm_scale * 1.4426950408889634f * qk_scale;
     // persistent: one thread block per SM (fewer when the list is shorter)
     const int sms = max_blocks > 0 ? std::min(max_blocks, pl->num_sms) : pl->num_sms;
     const unsigned grid = (unsigned)std::min<size_t>(n_work, (size_t)sms);
-    attn_tc_kernel<D, kMaxPages><<<grid, kThreads, Geo<D>::kSmemAlloc, st>>>(
+    attn_tc_kernel<D, kMaxPages, K8><<<grid, kThreads, Geo<D>::kSmemAlloc, st>>>(
         tq, tk, tv, to, d.tiles, work, (int)n_work, d.q_pos, d.page_off, d.pages, d.seq_len,
         static_cast<__nv_bfloat16 *>(out), lse, Hq, g, Hkv, ps, pl->num_pool_pages, scale_log2, pl->max_parts, d.ws_o, d.ws_ml, d.status);
     count_launch();
@@ -751,10 +770,22 @@ cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, c
         return cudaErrorNotSupported;
     }
     if (ps == 8)
-        return D == 128 ? launch_attn_tc_d<128, 16>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, st, err)
-                        : launch_attn_tc_d<64, 16>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, st, err);
-    return D == 128 ? launch_attn_tc_d<128, 8>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, st, err)
-                    : launch_attn_tc_d<64, 8>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, st, err);
+        return D == 128 ? launch_attn_tc_d<128, 16, false>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, 1.f, st, err)
+                        : launch_attn_tc_d<64, 16, false>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, 1.f, st, err);
+    return D == 128 ? launch_attn_tc_d<128, 8, false>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, 1.f, st, err)
+                    : launch_attn_tc_d<64, 8, false>(pl, k_pool, v_pool, q, out, lse, chunk, max_blocks, 1.f, st, err);
+}
+
+cudaError_t launch_attn_tc_k8(const tessera_plan *pl, void *k_pool8, void *v_pool, const void *q8, void *out,
+                              float *lse, float qk_scale, cudaStream_t st, std::string *err) {
+    if (pl->n_q == 0 || pl->work.empty()) return cudaSuccess;
+    const int D = pl->cfg.head_dim, ps = pl->cfg.page_size, g = pl->cfg.num_q_heads / pl->cfg.num_kv_heads;
+    if (D != 128 || (ps != 8 && ps != 16 && ps != 32 && ps != 64 && ps != 128) || g > 16) {
+        *err = "8-bit keys: head_dim 128 only";
+        return cudaErrorNotSupported;
+    }
+    return ps == 8 ? launch_attn_tc_d<128, 16, true>(pl, k_pool8, v_pool, q8, out, lse, -1, 0, qk_scale, st, err)
+                   : launch_attn_tc_d<128, 8, true>(pl, k_pool8, v_pool, q8, out, lse, -1, 0, qk_scale, st, err);
 }
 
 }  // namespace tessera

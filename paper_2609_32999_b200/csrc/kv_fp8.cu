@@ -12,6 +12,7 @@
 #include <cuda_fp8.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <type_traits>
 
 #include "launch.h"
@@ -187,6 +188,35 @@ kv_fp8_kernel(const void *__restrict__ k_src, const void *__restrict__ v_src, vo
     }
 }
 
+// bf16 -> e4m3 codes of (value * mul): 8 elements per thread, grid-stride.
+__global__ void __launch_bounds__(256)
+quantize_e4m3_kernel(const uint4 *__restrict__ src, uint2 *__restrict__ dst, int64_t n_chunks, float mul) {
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_chunks; e += (int64_t)gridDim.x * blockDim.x) {
+        float f[8];
+        unpack_bf16x8(__ldg(src + e), f);
+        dst[e] = pack_e4m3x8(f, mul);
+    }
+}
+
+// Fresh rows of the recompute tokens into an 8-bit key pool and a 16-bit value pool (Sec. 5.3: recomputed
+// states override cached ones): K as the e4m3 code of (k * k_mul), V as a bit copy.
+__global__ void __launch_bounds__(256)
+scatter_fresh_k8_kernel(uint2 *__restrict__ k_pool8, uint4 *__restrict__ v_pool, const uint4 *__restrict__ k_new,
+                        const uint4 *__restrict__ v_new, const int32_t *__restrict__ fresh_dst, int64_t n_chunks,
+                        int row_chunks, float k_mul) {
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n_chunks; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t j = e / row_chunks;
+        const int c = (int)(e - j * row_chunks);
+        const size_t o = (size_t)fresh_dst[j] * row_chunks + c;
+        if (k_new) {
+            float f[8];
+            unpack_bf16x8(__ldg(k_new + e), f);
+            k_pool8[o] = pack_e4m3x8(f, k_mul);
+        }
+        if (v_new) v_pool[o] = __ldg(v_new + e);
+    }
+}
+
 template <int D, bool TO_8BIT, bool IL>
 cudaError_t launch_d(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst, bool rotate,
                      float k_mul, float v_mul, const int32_t *g_src, int first_item, int n, int max_blocks, cudaStream_t st) {
@@ -215,6 +245,28 @@ cudaError_t launch_dir(const tessera_plan *pl, const void *k_src, const void *v_
 }
 
 }  // namespace
+
+cudaError_t launch_quantize_e4m3(const void *src_bf16, void *dst8, int64_t n_elems, float mul, cudaStream_t st) {
+    const int64_t n_chunks = n_elems / 8;
+    if (n_chunks == 0) return cudaSuccess;
+    const int blocks = (int)std::min<int64_t>((n_chunks + 255) / 256, 148 * 16);
+    quantize_e4m3_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4 *>(src_bf16), static_cast<uint2 *>(dst8), n_chunks, mul);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scatter_fresh_k8(const tessera_plan *pl, void *k_pool8, void *v_pool, const void *k_new,
+                                    const void *v_new, float k_mul, cudaStream_t st) {
+    if (pl->n_q == 0 || (!k_new && !v_new)) return cudaSuccess;
+    const int row_chunks = pl->cfg.num_kv_heads * pl->cfg.head_dim / 8;
+    const int64_t n_chunks = pl->n_q * row_chunks;
+    const int blocks = (int)std::min<int64_t>((n_chunks + 255) / 256, (int64_t)pl->num_sms * 16);
+    scatter_fresh_k8_kernel<<<blocks, 256, 0, st>>>(static_cast<uint2 *>(k_pool8), static_cast<uint4 *>(v_pool),
+                                                   static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new),
+                                                   pl->dev.fresh_dst, n_chunks, row_chunks, k_mul);
+    count_launch();
+    return cudaGetLastError();
+}
 
 cudaError_t launch_kv_fp8_range(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst, void *v_dst,
                                 bool to_8bit, bool rotate, float k_mul, float v_mul, const int32_t *g_src, int first_item,

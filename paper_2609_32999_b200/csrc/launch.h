@@ -43,4 +43,14 @@ cudaError_t launch_scatter_fresh(const tessera_plan *pl, void *k_pool, void *v_p
 cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, const void *q, void *out,
                            float *lse, int chunk, int max_blocks, cudaStream_t st, std::string *err);
 
+// The same kernel with 8-bit (e4m3) queries and keys: q8 [n_q][H_q][D] and k_pool8 hold codes, qk_scale is the
+// product of their two scales; head_dim 128 only; the whole batch on the full grid.
+cudaError_t launch_attn_tc_k8(const tessera_plan *pl, void *k_pool8, void *v_pool, const void *q8, void *out,
+                              float *lse, float qk_scale, cudaStream_t st, std::string *err);
+// bf16 rows -> e4m3 codes of (value * mul), nearest-even, saturating: n_elems elements (a multiple of 8).
+cudaError_t launch_quantize_e4m3(const void *src_bf16, void *dst8, int64_t n_elems, float mul, cudaStream_t st);
+// Fresh rows into an 8-bit key pool (codes of k_new * k_mul) and a 16-bit value pool (bit copies).
+cudaError_t launch_scatter_fresh_k8(const tessera_plan *pl, void *k_pool8, void *v_pool, const void *k_new,
+                                    const void *v_new, float k_mul, cudaStream_t st);
+
 }  // namespace tessera

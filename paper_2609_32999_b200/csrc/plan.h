@@ -66,6 +66,7 @@ struct DeviceTables {
     int32_t *status = nullptr;     // device status word(s)
     double *inv_freq = nullptr;    // [D/2] rotary frequencies
     // staging for the host-buffer entry point (allocated on first use)
+    void *q8 = nullptr;            // 8-bit copy of q for the 8-bit-key attention entry (allocated on first use)
     void *st_q = nullptr, *st_k = nullptr, *st_v = nullptr, *st_o = nullptr;
     float *st_lse = nullptr;
 };

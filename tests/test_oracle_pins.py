@@ -343,6 +343,32 @@ def test_attention_brute_force_tiny():
             assert abs(math.log(z) - lse[j, h]) < 1e-12
 
 
+def test_attention_with_float64_queries_against_numpy_softmax():
+    """The fp64-query form of the oracle's attention (used for 8-bit-key attention, whose decoded queries
+    need not be bf16 numbers): brute force with numpy on a tiny case, and equal to the bf16-query form
+    when the queries are bf16 numbers."""
+    shape = wl.ModelShape(4, 2, 8, 4, 1e4)
+    rng = np.random.default_rng(12)
+    T = 19
+    w = wl.build_workload("q64", shape, [[wl.unit(T, "a", cached=False)]], rng)
+    k = rng.standard_normal((T, 2, 8))
+    v = torch.from_numpy(rng.standard_normal((T, 2, 8))).to(torch.bfloat16)
+    q = rng.standard_normal((T, 4, 8)) * 0.37                                  # not bf16 numbers
+    jj, hh, pp = orc.request_rows(w, 0)
+    o, l = orc.attention_rows(w, k, orc.bits(v), q, jj, hh, pp)
+    vd = v.double().numpy()
+    for i in range(len(jj)):
+        p, h = int(pp[i]), int(hh[i])
+        sc = (k[: p + 1, h // 2] @ q[jj[i], h]) / math.sqrt(8)
+        wgt = np.exp(sc - sc.max()); wgt /= wgt.sum()
+        assert np.max(np.abs(o[i] - wgt @ vd[: p + 1, h // 2])) < 1e-12
+        assert abs(l[i] - (sc.max() + math.log(np.exp(sc - sc.max()).sum()))) < 1e-12
+    qb = torch.from_numpy(q).to(torch.bfloat16)
+    o1, l1 = orc.attention_rows(w, k, orc.bits(v), orc.bits(qb), jj, hh, pp)
+    o2, l2 = orc.attention_rows(w, k, orc.bits(v), qb.double().numpy(), jj, hh, pp)
+    assert np.array_equal(o1, o2) and np.array_equal(l1, l2)
+
+
 def test_partial_equals_rows_of_library_causal_attention():
     """Recompute set = all tokens reproduces ordinary causal prefill (library SDPA,
     fp64, KV heads repeated g times); any subset equals the matching rows."""
