@@ -297,8 +297,8 @@ TESSERA_API int32_t tessera_partial_prefill_attn(const tessera_plan *plan, void 
  * value 448), S = Q K^T runs on the 8-bit tensor-core path, probabilities, values and the accumulator stay
  * as in tessera_partial_prefill_attn.
  *   k_pool8   device [num_pool_pages][page_size][H_kv][D] bytes: code c stands for c * k_scale.  The
- *             request's destination pages must hold its assembled keys as codes (e.g. written by
- *             tessera_kv_retain_fp8 with a compose plan, which rotates and quantises on the way).
+ *             request's destination pages must hold its assembled keys as codes (written by
+ *             tessera_kv_compose_k8, which rotates and quantises on the way).
  *   v_pool    device, 16-bit pool as everywhere else
  *   q         device [n_q][H_q][D] bf16, already rotated; quantised by the call itself into a buffer the
  *             plan owns (allocated on the first call): code = e4m3_rne(q * fp32(1 / q_scale)), saturating
@@ -309,6 +309,16 @@ TESSERA_API int32_t tessera_partial_prefill_attn(const tessera_plan *plan, void 
  * over the DECODED operands (the codes times their scales) at the usual tolerance: the quantisation is
  * part of the method, not an error of the kernel.
  */
+/*
+ * Companion of the call below: "preparing cache hits" (Sec. 5.3) for the 8-bit-key attention path.  Like
+ * tessera_kv_compose_from (16-bit units in a separate source pool, desc.num_source_pages > 0), but the
+ * key rows land in the 8-bit pool k_pool8 - rotated (with TESSERA_FUSE_ROPE) in fp32, multiplied by
+ * fp32(1 / k_scale) and rounded to the nearest e4m3 code, ties to even, saturating - while the value rows
+ * are bit copies into the 16-bit v_pool.  No counterpart in the paper.  One kernel; nothing is allocated.
+ */
+TESSERA_API int32_t tessera_kv_compose_k8(const tessera_plan *plan, const void *k_src, const void *v_src, void *k_pool8,
+                                          void *v_pool, float k_scale, uint32_t flags, void *stream);
+
 TESSERA_API int32_t tessera_partial_prefill_attn_k8(tessera_plan *plan, void *k_pool8, float k_scale, void *v_pool,
                                                     const void *q, float q_scale, const void *k_new, const void *v_new,
                                                     void *out, float *lse, void *stream);

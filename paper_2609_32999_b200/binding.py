@@ -55,7 +55,7 @@ class PlanInfo(ctypes.Structure):
 
 
 EXPORTS = ["tessera_plan_create", "tessera_plan_destroy", "tessera_plan_block_table", "tessera_plan_get_info",
-           "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_kv_compose_from_fp8", "tessera_kv_retain_fp8", "tessera_rope_shift", "tessera_rope_fresh", "tessera_extend_write", "tessera_partial_prefill_attn", "tessera_partial_prefill_attn_k8",
+           "tessera_plan_status", "tessera_kv_compose", "tessera_kv_compose_from", "tessera_kv_compose_from_fp8", "tessera_kv_retain_fp8", "tessera_rope_shift", "tessera_rope_fresh", "tessera_extend_write", "tessera_partial_prefill_attn", "tessera_kv_compose_k8", "tessera_partial_prefill_attn_k8",
            "tessera_composed_prefill_host", "tessera_composed_prefill_host_tier", "tessera_rope_shift_static", "tessera_selftest_bounded_wait", "tessera_last_error",
            "tessera_launch_count"]
 
@@ -74,6 +74,7 @@ _lib.tessera_rope_shift.argtypes = [_vp, _vp, _vp]
 _lib.tessera_rope_fresh.argtypes = [_vp, _vp, _vp, _vp]
 _lib.tessera_extend_write.argtypes = [_vp] * 9
 _lib.tessera_partial_prefill_attn.argtypes = [_vp] * 9
+_lib.tessera_kv_compose_k8.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_float, ctypes.c_uint32, _vp]
 _lib.tessera_partial_prefill_attn_k8.argtypes = [_vp, _vp, ctypes.c_float, _vp, _vp, ctypes.c_float, _vp, _vp, _vp, _vp, _vp]
 _lib.tessera_composed_prefill_host.argtypes = [_vp] * 9
 _lib.tessera_composed_prefill_host_tier.argtypes = [_vp, _vp, _vp, ctypes.c_int32, ctypes.c_float, ctypes.c_float,
@@ -219,6 +220,11 @@ class Plan:
     def partial_prefill_attn(self, k_pool, v_pool, q, k_new, v_new, out, lse=None, stream=None) -> None:
         _check(_lib.tessera_partial_prefill_attn(self._h, _dev(k_pool), _dev(v_pool), _dev(q), _dev(k_new),
                                                  _dev(v_new), _dev(out), _dev(lse), _stream(stream)))
+
+    def kv_compose_k8(self, k_src, v_src, k_pool8, v_pool, k_scale: float, fuse_rope: bool = True, stream=None) -> None:
+        """16-bit source pools -> keys as e4m3 codes in k_pool8 (rotated on the way), values into the 16-bit v_pool."""
+        _check(_lib.tessera_kv_compose_k8(self._h, _dev(k_src), _dev(v_src), _dev(k_pool8), _dev(v_pool), float(k_scale),
+                                          FUSE_ROPE if fuse_rope else 0, _stream(stream)))
 
     def partial_prefill_attn_k8(self, k_pool8, k_scale: float, v_pool, q, q_scale: float, k_new, v_new, out, lse=None,
                                 stream=None) -> None:

@@ -336,6 +336,14 @@ int32_t tessera_kv_retain_fp8(const tessera_plan *pl, const void *k_src, const v
     return TESSERA_OK;
 }
 
+int32_t tessera_kv_compose_k8(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_pool8, void *v_pool,
+                              float k_scale, uint32_t flags, void *stream) {
+    if (int32_t rc = check_fp8_call(pl, k_src, v_src, k_pool8, v_pool, flags, k_scale, 1.0f)) return rc;
+    TS_CUDA(launch_compose_k8(pl, k_src, v_src, k_pool8, v_pool, (flags & TESSERA_FUSE_ROPE) != 0, 1.0f / k_scale,
+                              static_cast<cudaStream_t>(stream)));
+    return TESSERA_OK;
+}
+
 int32_t tessera_rope_shift(const tessera_plan *pl, void *k_pool, void *stream) {
     if (int32_t rc = check_device_plan(pl)) return rc;
     if (!k_pool || misaligned(k_pool)) return set_error(TESSERA_INVALID_ARG, "k_pool must be non-null and 16-byte aligned");

@@ -94,8 +94,10 @@ __device__ __forceinline__ int cs_index(int c, int i) {
 }
 
 // One thread block per GatherItem.  TO_8BIT false: sources are e4m3 (mul = scale), destinations bf16;
-// TO_8BIT true: sources are bf16, destinations e4m3 (mul = 1 / scale, applied after the rotation).
-template <int D, bool TO_8BIT, bool ROTATE, bool INTERLEAVED>
+// TO_8BIT true: sources are bf16, destinations e4m3 (mul = 1 / scale, applied after the rotation); with V16
+// only the keys go 8-bit and the value rows are bit copies into a 16-bit pool (key pages for the 8-bit
+// attention path, values as everywhere else).
+template <int D, bool TO_8BIT, bool ROTATE, bool INTERLEAVED, bool V16 = false>
 __global__ void __launch_bounds__(kThreads)
 kv_fp8_kernel(const void *__restrict__ k_src, const void *__restrict__ v_src, void *__restrict__ k_dst,
               void *__restrict__ v_dst, const int32_t *__restrict__ g_src, const int32_t *__restrict__ g_dst,
@@ -170,11 +172,18 @@ kv_fp8_kernel(const void *__restrict__ k_src, const void *__restrict__ v_src, vo
                 rotate_f<INTERLEAVED>(klo, khi, cr);
             }
             if constexpr (TO_8BIT) {
-                uint2 *kd = static_cast<uint2 *>(k_dst), *vd = static_cast<uint2 *>(v_dst);
+                uint2 *kd = static_cast<uint2 *>(k_dst);
                 kd[dso[u]] = pack_e4m3x8(klo, k_mul);
                 kd[dso[u] + HALF] = pack_e4m3x8(khi, k_mul);
-                vd[dso[u]] = pack_e4m3x8(vlo, v_mul);
-                vd[dso[u] + HALF] = pack_e4m3x8(vhi, v_mul);
+                if constexpr (V16) {
+                    uint4 *vd = static_cast<uint4 *>(v_dst);
+                    vd[dso[u]] = rv[u][0];
+                    vd[dso[u] + HALF] = rv[u][1];
+                } else {
+                    uint2 *vd = static_cast<uint2 *>(v_dst);
+                    vd[dso[u]] = pack_e4m3x8(vlo, v_mul);
+                    vd[dso[u] + HALF] = pack_e4m3x8(vhi, v_mul);
+                }
             } else {
                 uint4 *kd = static_cast<uint4 *>(k_dst), *vd = static_cast<uint4 *>(v_dst);
                 kd[dso[u]] = pack_bf16x8(klo);
@@ -245,6 +254,28 @@ cudaError_t launch_dir(const tessera_plan *pl, const void *k_src, const void *v_
 }
 
 }  // namespace
+
+// Keys rotated and quantised into an 8-bit pool, values copied into a 16-bit pool (sources 16-bit).
+cudaError_t launch_compose_k8(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst8, void *v_dst,
+                              bool rotate, float k_mul, cudaStream_t st) {
+    const int n = (int)pl->items.size();
+    if (n == 0) return cudaSuccess;
+    const DeviceTables &d = pl->dev;
+    const int H = pl->cfg.num_kv_heads;
+    const bool il = pl->cfg.rope_pairing == 1;
+#define TESSERA_K8_LAUNCH(DD, ROT, IL) \
+    kv_fp8_kernel<DD, true, ROT, IL, true><<<n, kThreads, 0, st>>>(k_src, v_src, k_dst8, v_dst, d.g_src, d.g_dst, d.items, n, d.rope, H, k_mul, 1.f)
+    if (pl->cfg.head_dim == 128) {
+        if (rotate) { if (il) TESSERA_K8_LAUNCH(128, true, true); else TESSERA_K8_LAUNCH(128, true, false); }
+        else { if (il) TESSERA_K8_LAUNCH(128, false, true); else TESSERA_K8_LAUNCH(128, false, false); }
+    } else {
+        if (rotate) { if (il) TESSERA_K8_LAUNCH(64, true, true); else TESSERA_K8_LAUNCH(64, true, false); }
+        else { if (il) TESSERA_K8_LAUNCH(64, false, true); else TESSERA_K8_LAUNCH(64, false, false); }
+    }
+#undef TESSERA_K8_LAUNCH
+    count_launch();
+    return cudaGetLastError();
+}
 
 cudaError_t launch_quantize_e4m3(const void *src_bf16, void *dst8, int64_t n_elems, float mul, cudaStream_t st) {
     const int64_t n_chunks = n_elems / 8;

@@ -47,6 +47,10 @@ cudaError_t launch_attn_tc(const tessera_plan *pl, void *k_pool, void *v_pool, c
 // product of their two scales; head_dim 128 only; the whole batch on the full grid.
 cudaError_t launch_attn_tc_k8(const tessera_plan *pl, void *k_pool8, void *v_pool, const void *q8, void *out,
                               float *lse, float qk_scale, cudaStream_t st, std::string *err);
+// Compose for the 8-bit-key attention path: 16-bit sources -> keys (rotated, times k_mul) as e4m3 codes in
+// k_dst8, values as bit copies in the 16-bit v_dst.
+cudaError_t launch_compose_k8(const tessera_plan *pl, const void *k_src, const void *v_src, void *k_dst8, void *v_dst,
+                              bool rotate, float k_mul, cudaStream_t st);
 // bf16 rows -> e4m3 codes of (value * mul), nearest-even, saturating: n_elems elements (a multiple of 8).
 cudaError_t launch_quantize_e4m3(const void *src_bf16, void *dst8, int64_t n_elems, float mul, cudaStream_t st);
 // Fresh rows into an 8-bit key pool (codes of k_new * k_mul) and a 16-bit value pool (bit copies).
