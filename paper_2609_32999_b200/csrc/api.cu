@@ -259,7 +259,7 @@ int32_t tessera_plan_get_info(const tessera_plan *pl, tessera_plan_info *info) {
     info->attn_flops = 4LL * pl->cfg.head_dim * pl->cfg.num_q_heads * pl->qk_pairs;
     info->n_rope_rows = (int32_t)pl->rope_delta.size();
     info->n_gather_items = (int32_t)pl->items.size();
-    info->n_attn_items = (int32_t)pl->work.size();
+    info->n_attn_items = pl->n_work_items;
     info->attn_kernel = pl->attn_kernel;
     info->retained_tokens = pl->retained_tokens;
     info->attn_mma_pairs = pl->mma_pairs;

@@ -145,12 +145,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const int pps = kStep / page_size;                 // pages per step: 1, 2, 4, 8 or 16
 
     // The block's share of the work list: round k of the grid takes items [k G, (k + 1) G), this block
-    // the b-th of them in even rounds and the b-th from the end in odd rounds (the list is sorted by
-    // cost, so the serpentine evens out the sums; blocks that run at the same time work on neighbours
-    // in the list, i.e. on the same request and KV head, and share their K/V pages in L2.  A greedy
-    // least-loaded assignment computed on the host balanced the modelled cost better and measured
-    // 0.5-2 % slower; taking items off a global counter at run time measured 1-1.5 % slower on the
-    // long-context configurations).  Every role walks the same sequence; -1 = nothing in this round.
+    // the b-th of them in even rounds and the b-th from the end in odd rounds.  For a list sorted by
+    // cost the serpentine evens out the sums, and blocks that run at the same time work on neighbours
+    // in the list, i.e. on the same request and KV head, and share their K/V pages in L2.  When a batch
+    // has few items per block the host lays the list out so that this very walk hands each block a
+    // greedily balanced share (holes are marked tile_a = -1).  Taking items off a global counter at
+    // run time measured 1-1.5 % slower on the long-context configurations.  Every role walks the
+    // same sequence; -1 = nothing in this round.
     const int n_rounds = (n_work + (int)gridDim.x - 1) / (int)gridDim.x;
     auto item_index = [&](int round) {
         const int b = (round & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;
@@ -160,6 +161,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     auto load_item = [&](int w) {
         Item it;
         it.wk = work[w];
+        if (it.wk.tile_a < 0) {            // a hole of the assignment: nothing to do in this round
+            it.n_tiles = 0;
+            return it;
+        }
         it.n_tiles = it.wk.tile_b >= 0 ? 2 : 1;
         it.t0 = tiles[it.wk.tile_a];
         it.t1 = tiles[it.n_tiles == 2 ? it.wk.tile_b : it.wk.tile_a];
@@ -237,6 +242,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             const int w = item_index(round);
             if (w < 0) continue;
             const Item it = load_item(w);
+            if (it.n_tiles == 0) continue;
             const int kvh = it.wk.kvh;
             if (lane == 0) {
                 for (int q = 0; q < it.n_tiles; ++q) {
@@ -303,6 +309,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             const int w = item_index(round);
             if (w < 0) continue;
             const Item it = load_item(w);
+            if (it.n_tiles == 0) continue;
             const int n_steps = it.n_steps;
             const int my_steps = q ? it.n_steps1 : it.n_steps0;
             const int T = it.T, step0 = it.step0;
@@ -437,6 +444,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         const int w = item_index(round);
         if (w < 0) continue;
         const Item it = load_item(w);
+        if (it.n_tiles == 0) continue;
         const int n_tiles = it.n_tiles, n_steps = it.n_steps, n_steps0 = it.n_steps0, n_steps1 = it.n_steps1;
         const int step0 = it.step0, kvh = it.wk.kvh;
         const AttnTile &t0 = it.t0, &t1 = it.t1;

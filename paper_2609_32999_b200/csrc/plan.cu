@@ -413,6 +413,46 @@ int32_t build_plan_host(const tessera_model_cfg *cfg, const tessera_compose_desc
         // together, so thread blocks that run at the same time stream the same K/V pages and find
         // them in L2.
         sort_items(pl->work.begin(), pl->work.end());
+        // With few items per thread block the spread of the blocks' finishing times is what costs (config 3:
+        // 7 items per block, slowest block 8-10 % above the mean with the plain walk): the items are then
+        // assigned greedily to the least-loaded block by modelled cycles (item fetch 700, epilogue + first
+        // step 3 150 per tile, 3 180 per step of both tiles, 1 650 per step of one - measured with clock64)
+        // and laid out so that the kernel's serpentine walk (round k, block b -> index k G + (k odd ? G - 1
+        // - b : b)) hands every block its own list; holes are marked tile_a = -1.  Measured: config 3 +6 %,
+        // config 4 +-0.  With many items per block (config 5: 131) the plain walk is already even and keeps
+        // neighbours in the list - the same request and head - on the GPU at the same time, which the
+        // greedy assignment does not: it measured 3 % slower there, so it is not used.
+        auto lpt_layout = [&](std::vector<AttnWork> &list) {
+            const int G = num_sms;
+            if ((int)list.size() <= G || (int)list.size() > kLptMaxItemsPerBlock * G) return;
+            auto cycles = [&](const AttnWork &w) -> int64_t {
+                const int sa = std::min(w.step_end, steps_of(w.tile_a)) - w.step_begin;
+                const int sb = w.tile_b >= 0 ? std::min(w.step_end, steps_of(w.tile_b)) - w.step_begin : 0;
+                const int both = std::min(sa, sb), single = std::max(sa, sb) - both, nt = w.tile_b >= 0 ? 2 : 1;
+                return 700 + (int64_t)nt * 3150 + (int64_t)both * 3180 + (int64_t)single * 1650;
+            };
+            std::vector<int> order(list.size());
+            std::iota(order.begin(), order.end(), 0);
+            std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cycles(list[a]) > cycles(list[b]); });
+            std::vector<int64_t> load(G, 0);
+            std::vector<std::vector<int>> mine(G);
+            for (int i : order) {
+                const int b = (int)(std::min_element(load.begin(), load.end()) - load.begin());
+                load[b] += cycles(list[i]);
+                mine[b].push_back(i);
+            }
+            size_t rounds = 0;
+            for (auto &m : mine) rounds = std::max(rounds, m.size());
+            AttnWork hole{};
+            hole.tile_a = -1; hole.tile_b = -1;
+            std::vector<AttnWork> out(rounds * G, hole);
+            for (int b = 0; b < G; ++b)
+                for (size_t k = 0; k < mine[b].size(); ++k)
+                    out[k * G + ((k & 1) ? G - 1 - b : b)] = list[mine[b][k]];
+            list.swap(out);
+        };
+        pl->n_work_items = (int32_t)pl->work.size();
+        lpt_layout(pl->work);
     }
 
     pl->total_tokens = total;

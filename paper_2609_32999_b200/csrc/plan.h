@@ -17,6 +17,7 @@ constexpr int kDefaultSMs = 148;         // SM count assumed by a host-only plan
 constexpr int kSplitMinSteps = 4;        // never split below this many 128-key steps per part
 constexpr int kSplitMaxParts = 8;
 constexpr int kHostChunks = 4;          // request chunks of the host-buffer entry point's copy / compute pipeline
+constexpr int kLptMaxItemsPerBlock = 16;  // above this many attention items per thread block the plain serpentine walk is kept
 constexpr int kAttnCostBands = 16;      // cost bands of the attention work list (longest band first)
 
 // One thread block of the gather / shift kernel: `count` consecutive entries of the copy list that
@@ -102,6 +103,7 @@ struct tessera_plan {
     std::vector<int32_t> chunk_item_off;                  // [n_chunks + 1]; gather items of the chunk's requests
     std::vector<tessera::CombineItem> combine;     // grouped by chunk: [chunk_combine_off[c], chunk_combine_off[c+1])
     std::vector<int32_t> chunk_combine_off;
+    int32_t n_work_items = 0;                      // real items of `work` (the list may hold holes)
     int32_t max_parts = 1;                         // split-KV parts per item (1 = no split)
     int32_t attn_kernel = 0;
     int32_t tile_tokens = 0;
