@@ -21,14 +21,24 @@
  *                           even and saturation.  The paper stores conventional 16-bit K/V
  *                           (Sec. 8); the 8-bit tier is this build's extension and these two
  *                           functions are its definition.
+ *   oracle_f64_to_bf16_rne - one round-to-nearest-even of a double to bf16 (how an expanded
+ *                           8-bit row is defined: the exact product code x scale, rounded once).
  *   oracle_attention_rows - the extend pass restricted to the recompute rows
  *                           (Sec. 5.3, Sec. 6.1 "Implementation"): causal softmax
  *                           attention of a query at position p over keys 0..p.
+ *   oracle_attention_rows_qf64 - the same with the queries given as doubles (decoded 8-bit
+ *                           queries of this build's 8-bit-key attention).
+ *   oracle_assemble_ex(.., fresh_k_raw) - fresh keys handed over before rotation (Sec. 6.1: the
+ *                           forward path captures pre-RoPE keys): the request sees them rotated
+ *                           for their positions.
  *
  * Pins (tests/test_oracle_pins.py): composition and relative-position identities,
- * one-hot closed form, a library rotary routine, a 2-D rotation matrix, the
- * paper's worked position example, brute-force attention, library causal
- * attention, uniform-softmax closed form, per-token placement loop.
+ * one-hot closed form, a library rotary routine (also for the fresh_k_raw branch), a 2-D
+ * rotation matrix, the paper's worked position example, brute-force attention (bf16 and
+ * fp64 queries), library causal attention, uniform-softmax closed form, per-token placement
+ * loop and hand-worked slot numbers (tests/golden/placement_slots.txt), the retained form
+ * R(-(p0 + i)) with one worked number, the library's e4m3 and bf16 conversions, exact
+ * rational arithmetic for the single rounding of code x scale.  No function is unpinned.
  */
 #include <math.h>
 #include <stdint.h>
