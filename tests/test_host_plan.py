@@ -50,6 +50,12 @@ def test_host_only_plan_refuses_device_calls():
                  lambda: plan.kv_retain_fp8(None, None, None, None, 1.0, 1.0, stream=0),
                  lambda: plan.kv_compose_from(None, None, None, None, stream=0),
                  lambda: plan.rope_shift(None, stream=0),
+                 lambda: plan.rope_fresh(None, None, stream=0),
+                 lambda: plan.extend_write(None, None, None, None, None, stream=0),
+                 lambda: plan.kv_compose_k8(None, None, None, None, 1.0, stream=0),
+                 lambda: plan.partial_prefill_attn_k8(None, 1.0, None, None, 1.0, None, None, None, stream=0),
+                 lambda: plan.composed_prefill_host_tier(None, None, None, None, None, None, None, None, stream=0),
+                 lambda: plan.composed_prefill_host(None, None, None, None, None, None, stream=0),
                  lambda: plan.partial_prefill_attn(None, None, None, None, None, None, None, stream=0)):
         with pytest.raises(tb.TesseraError) as e:
             call()
